@@ -1,0 +1,211 @@
+/*
+ * rmsmp.h -- C ABI of the B200 (sm_100a) RMSMP layer library.
+ *
+ * The library runs the inference arithmetic of one linear or convolution layer quantized
+ * the RMSMP way (paper Section 3): every weight row (= output feature / filter) carries
+ * its own scheme and precision -- Power-of-Two 4-bit, Fixed-point 4-bit or Fixed-point
+ * 8-bit, in a per-layer ratio fixed offline -- and multiplies 4-bit fixed-point
+ * activations.  Integer accumulation is exact; the output is rescaled per row.
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller owns every
+ *     buffer; the library allocates no device memory and keeps no reference after a call
+ *     returns (work already queued on the stream keeps using the buffers until it is done).
+ *   - `stream` is a cudaStream_t passed as void* (0 = default stream).  All device work is
+ *     asynchronous on it.
+ *   - Every function returns an rmsmp_status and never throws, aborts or prints.  Everything
+ *     that can be validated on the host is validated before anything is launched.
+ *   - Device pointers must be 16-byte aligned unless stated otherwise.
+ */
+#ifndef RMSMP_H_
+#define RMSMP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RMSMP_OK = 0,
+    RMSMP_ERR_NULL = 1,             /* a required pointer is NULL */
+    RMSMP_ERR_SHAPE = 2,            /* a dimension is < 1 or beyond the supported range */
+    RMSMP_ERR_SCHEME = 3,           /* (scheme, bits) not one of PoT-4, Fixed-4, Fixed-8 */
+    RMSMP_ERR_SCALE = 4,            /* a clip value alpha is not finite and > 0 */
+    RMSMP_ERR_ALIGN = 5,            /* pointer or leading dimension not 16-byte aligned */
+    RMSMP_ERR_BUFFER_TOO_SMALL = 6, /* packed buffer smaller than rmsmp_layer.packed_bytes */
+    RMSMP_ERR_ARCH = 7,             /* current device is not compute capability 10.x */
+    RMSMP_ERR_CUDA = 8,             /* a CUDA runtime/driver call failed */
+    RMSMP_ERR_TIMEOUT = 9,          /* a bounded in-kernel wait ran out (device status word) */
+    RMSMP_ERR_BAD_LAYER = 10,       /* rmsmp_layer not produced by rmsmp_layer_init */
+    RMSMP_ERR_VARIANT = 11          /* requested kernel variant cannot run this problem */
+} rmsmp_status;
+
+/* The scheme/precision menu of the method (Figure 2): bits is 4 or 8; PoT only with 4. */
+typedef enum { RMSMP_SCHEME_POT = 0, RMSMP_SCHEME_FIXED = 1 } rmsmp_scheme;
+/* Activation codes: unsigned 4-bit (0..15, post-ReLU inputs) or symmetric signed (-7..7). */
+typedef enum { RMSMP_ACT_U4 = 0, RMSMP_ACT_S4 = 1 } rmsmp_act_kind;
+/* PoT rounding: nearest level of Eq. 4 (default) or the printed 2^round(log2 x) rule of Eq. 5. */
+typedef enum { RMSMP_POT_NEAREST = 0, RMSMP_POT_LOG2 = 1 } rmsmp_pot_mode;
+/* Output layout: y[n*ld + m] (pixels/tokens major, default) or y[m*ld + n]. */
+typedef enum { RMSMP_OUT_NM = 0, RMSMP_OUT_MN = 1 } rmsmp_out_layout;
+/* Weight source layout: [M][K] row-major, or filters [M][Cin][kh][kw]. */
+typedef enum { RMSMP_W_LINEAR = 0, RMSMP_W_CONV_OIHW = 1 } rmsmp_w_layout;
+/* Which kernel carries out the contraction. */
+typedef enum {
+    RMSMP_VARIANT_AUTO = 0,      /* library picks by shape */
+    RMSMP_VARIANT_TENSOR = 1,    /* TMA + in-smem code expansion + tcgen05 int8 MMA, TMEM accumulators */
+    RMSMP_VARIANT_SIMT = 2,      /* CUDA-core integer multiply-add (dp4a) on codes expanded in registers */
+    RMSMP_VARIANT_SHIFTADD = 3,  /* CUDA cores; PoT rows by shift-and-add, no multiplier */
+    RMSMP_VARIANT_SIMPLE = 4     /* one thread per output, scalar; bring-up / cross-check */
+} rmsmp_variant;
+
+/*
+ * Host-side description of one packed layer.  Filled by rmsmp_layer_init from the shape and
+ * the per-row scheme map; plain data, may be copied or stored with the packed buffer.
+ * The packed buffer itself is position independent.
+ *
+ * Packed buffer layout (offsets in bytes from its start, every section 256-byte aligned):
+ *   header (256 B: magic, version, dims, counts; device status word at byte 64)
+ *   perm  [M] int32   packed position -> original row; PoT-4 rows, then Fixed-4, then
+ *                     Fixed-8, each group in original order (stable)
+ *   slot  [M] int32   original row -> packed position
+ *   wstep [M] float   by original row: real weight = integer value * wstep
+ *   alpha [M] float   by original row: clip value used by the quantizer
+ *   kind  [M] uint8   by original row: 0 PoT-4, 1 Fixed-4, 2 Fixed-8
+ *   blocks[ceil(M/128)][8] int32: for each block of 128 original rows the first packed
+ *                     position and count of its PoT-4, Fixed-4 and Fixed-8 rows
+ *                     {p0, nP, f0, nF, e0, nE, 0, 0} (positions relative to each group)
+ *   q4    [(nP+nF4)][Kp/2] bytes: 4-bit codes, two per byte
+ *   q8    [n8][Kp] bytes: int8 codes
+ * Reduction index inside a packed row: k' = (i*kw + j)*Cp + c  (tap-major, channels last),
+ * Cp = Cin rounded up to 32, Kp = kh*kw*Cp rounded up to 128; pad codes are zero.
+ * Inside each aligned group of 32 codes (16 bytes): PoT-4 stores code 2b in the low and
+ * 2b+1 in the high nibble of byte b (nibble = sign<<3 | e, value 0 or +-2^(e-1));
+ * Fixed-4 stores code b in the high and code 16+b in the low nibble of byte b
+ * (two's complement).
+ */
+typedef struct rmsmp_layer {
+    uint32_t magic;             /* set by rmsmp_layer_init */
+    int32_t M, Cin, kh, kw;     /* rows; reduction length K = Cin*kh*kw (linear: kh = kw = 1) */
+    int32_t Cp, Kp;             /* padded channel count per tap, padded packed row length */
+    int32_t nP, nF4, n8;        /* rows per group */
+    int32_t nblocks;            /* ceil(M/128) */
+    int32_t reserved;
+    uint64_t off_perm, off_slot, off_wstep, off_alpha, off_kind, off_blocks, off_q4, off_q8;
+    uint64_t packed_bytes;      /* size the packed buffer must have */
+} rmsmp_layer;
+
+const char* rmsmp_status_string(rmsmp_status s);
+
+/*
+ * Host helper: scheme/precision map of a layer from the ratio PoT-4 : Fixed-4 : Fixed-8 =
+ * A : B : C (Section 3.3, A + B + C = 100; Section 3.1: lower variance -> PoT).
+ * n8 = floor(M*C/100 + 1/2) rows of HIGHEST variance get Fixed-8 (a stand-in for the
+ * Hessian ranking of Algorithm 1, which needs a loss), of the rest the nP = floor(M*A/100
+ * + 1/2) rows of LOWEST variance get PoT-4, the others Fixed-4.  Ranking key: (population
+ * variance in double, row index).  h_W is [M][K] fp32 on the host; h_scheme / h_bits
+ * receive M entries.  Errors: NULL, SHAPE (M, K < 1 or A + B + C != 100 or negative).
+ */
+rmsmp_status rmsmp_assign_rows(const float* h_W, int M, int K, int A, int B, int C,
+                               uint8_t* h_scheme, uint8_t* h_bits);
+
+/*
+ * Describe a layer: counts rows per group, lays out the packed buffer, sets
+ * layer->packed_bytes.  Host only; no CUDA call.  Limits: 1 <= M <= 2^20,
+ * 1 <= Cin*kh*kw <= 1,000,000 (keeps |sum| < 2^31), kh, kw <= 16.
+ * Errors: NULL, SHAPE, SCHEME (an entry outside {PoT-4, Fixed-4, Fixed-8}; PoT-8 is not in
+ * the method, Section 3.2).
+ */
+rmsmp_status rmsmp_layer_init(rmsmp_layer* layer, int M, int Cin, int kh, int kw,
+                              const uint8_t* h_scheme, const uint8_t* h_bits);
+
+/*
+ * Quantize and pack the weights (Eq. 1-5; grouping by scheme, Section 3.1 / 4.1).
+ * d_W: fp32 weights on the device, [M][K] (RMSMP_W_LINEAR) or [M][Cin][kh][kw]
+ * (RMSMP_W_CONV_OIHW), 16-byte aligned.  h_scheme/h_bits/h_alpha: M host entries each
+ * (the assignment and the clip values are offline decisions).  Quantizers, per row r with
+ * t = clip(w / alpha_r, -1, 1) in fp32:
+ *   Fixed-m: q = round_half_even(t * (2^(m-1)-1)), weight = q * alpha_r/(2^(m-1)-1)
+ *   PoT-4:   sign/exponent code of the nearest level of +-{0, 2^-6..2^0} (ties to the larger
+ *            magnitude), or of 2^round(log2|t|) in RMSMP_POT_LOG2 mode; weight = v * alpha_r/64
+ * Writes layer->packed_bytes bytes to d_packed (256-byte aligned) and clears its status word.
+ * Errors: NULL, BAD_LAYER, SCHEME (map differs from the one given to rmsmp_layer_init),
+ * SCALE, ALIGN, BUFFER_TOO_SMALL, ARCH, CUDA.
+ */
+rmsmp_status rmsmp_quantize_pack(const float* d_W, rmsmp_w_layout w_layout,
+                                 const rmsmp_layer* layer, const uint8_t* h_scheme,
+                                 const uint8_t* h_bits, const float* h_alpha,
+                                 rmsmp_pot_mode pot_mode, void* d_packed, size_t packed_bytes,
+                                 void* stream);
+
+/*
+ * Parity/debug: expand a packed buffer back to integer values in ORIGINAL row order and
+ * original reduction order ([M][K], conv: [M][Cin][kh][kw]); Fixed rows give q, PoT rows
+ * 0 or +-2^(e-1).  d_perm (packed -> original, M int32) and d_wstep (by original row,
+ * M floats) may be NULL.  Errors: NULL, BAD_LAYER, ARCH, CUDA.
+ */
+rmsmp_status rmsmp_unpack_codes(const rmsmp_layer* layer, const void* d_packed,
+                                int8_t* d_values, int32_t* d_perm, float* d_wstep,
+                                void* stream);
+
+/*
+ * 4-bit activation quantizer (Section 3.1: activations are Fixed 4-bit for every row kind).
+ * One clip value per tensor.  U4: a = round_half_even(clip(x/alpha_a, 0, 1) * 15), step
+ * alpha_a/15.  S4: Fixed-4 of Eq. 1 with alpha_a, step alpha_a/7.  d_X: `count` floats;
+ * d_codes: `count` int8 (one code per byte).  *h_act_step receives the step (host, may be
+ * NULL).  Pointers need only their natural alignment.  Errors: NULL, SHAPE, SCALE, ARCH, CUDA.
+ */
+rmsmp_status rmsmp_quantize_act(const float* d_X, size_t count, float alpha_a,
+                                rmsmp_act_kind kind, int8_t* d_codes, float* h_act_step,
+                                void* stream);
+
+/*
+ * Linear layer (Algorithm 1, forward line): for every token n and row m
+ *   acc[n][m] = sum_k value[m][k] * act[n][k]          (int32, exact)
+ *   y[n][m]   = (float)acc[n][m] * (wstep[m] * act_step)
+ * d_act: int8 codes [N][ld_act], ld_act >= K and a multiple of 16.  d_out: fp32, layout
+ * `out_layout` with leading dimension ld_out (>= M for NM, >= N for MN).  d_acc (optional,
+ * may be NULL): int32 accumulators in the same layout and leading dimension.
+ * layer must describe a linear layer (kh = kw = 1).
+ * Errors: NULL, BAD_LAYER, SHAPE, ALIGN, ARCH, VARIANT, CUDA.
+ */
+rmsmp_status rmsmp_gemm(const rmsmp_layer* layer, const void* d_packed, const int8_t* d_act,
+                        int64_t N, int64_t ld_act, float act_step, float* d_out,
+                        int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
+                        void* stream);
+rmsmp_status rmsmp_gemm_variant(const rmsmp_layer* layer, const void* d_packed,
+                                const int8_t* d_act, int64_t N, int64_t ld_act, float act_step,
+                                float* d_out, int64_t ld_out, rmsmp_out_layout out_layout,
+                                int32_t* d_acc, rmsmp_variant variant, void* stream);
+
+/*
+ * Convolution layer as an implicit GEMM (no im2col buffer): activation codes d_act are
+ * [B][H][W][Cin] (channels last), zero outside the image; output pixel index
+ * n = (b*Ho + ho)*Wo + wo with Ho = (H + 2*pad - kh)/stride + 1 (same for Wo); results as in
+ * rmsmp_gemm with N = B*Ho*Wo and dense leading dimension (M for NM, N for MN).
+ * Errors: NULL, BAD_LAYER, SHAPE, ALIGN (Cin not a multiple of 16 for the tensor variant
+ * selects another variant under AUTO, and is VARIANT when RMSMP_VARIANT_TENSOR is forced),
+ * ARCH, VARIANT, CUDA.
+ */
+rmsmp_status rmsmp_conv_implicit(const rmsmp_layer* layer, const void* d_packed,
+                                 const int8_t* d_act, int B, int H, int W, int stride, int pad,
+                                 float act_step, float* d_out, rmsmp_out_layout out_layout,
+                                 int32_t* d_acc, void* stream);
+rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* layer, const void* d_packed,
+                                         const int8_t* d_act, int B, int H, int W, int stride,
+                                         int pad, float act_step, float* d_out,
+                                         rmsmp_out_layout out_layout, int32_t* d_acc,
+                                         rmsmp_variant variant, void* stream);
+
+/*
+ * Read the device status word of a packed buffer (synchronises the stream).  Kernels never
+ * trap: a bounded wait that runs out stores RMSMP_ERR_TIMEOUT there and the kernel returns.
+ */
+rmsmp_status rmsmp_last_device_status(const void* d_packed, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RMSMP_H_ */

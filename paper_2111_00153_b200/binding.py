@@ -1,0 +1,208 @@
+"""Thin ctypes binding of librmsmp.so: same names as include/rmsmp.h, argument marshalling only.
+
+Device buffers are torch CUDA tensors (or raw integer device pointers); torch is used for
+memory and streams, every step of the computation runs in the library's kernels.  There is no
+CPU fallback: if the library cannot be loaded, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librmsmp.so")
+
+# enums of rmsmp.h
+OK = 0
+SCHEME_POT, SCHEME_FIXED = 0, 1
+ACT_U4, ACT_S4 = 0, 1
+POT_NEAREST, POT_LOG2 = 0, 1
+OUT_NM, OUT_MN = 0, 1
+W_LINEAR, W_CONV_OIHW = 0, 1
+VARIANT_AUTO, VARIANT_TENSOR, VARIANT_SIMT, VARIANT_SHIFTADD, VARIANT_SIMPLE = 0, 1, 2, 3, 4
+(ERR_NULL, ERR_SHAPE, ERR_SCHEME, ERR_SCALE, ERR_ALIGN, ERR_BUFFER_TOO_SMALL, ERR_ARCH, ERR_CUDA,
+ ERR_TIMEOUT, ERR_BAD_LAYER, ERR_VARIANT) = range(1, 12)
+
+EXPORTS = (
+    "rmsmp_status_string", "rmsmp_assign_rows", "rmsmp_layer_init", "rmsmp_quantize_pack",
+    "rmsmp_unpack_codes", "rmsmp_quantize_act", "rmsmp_gemm", "rmsmp_gemm_variant",
+    "rmsmp_conv_implicit", "rmsmp_conv_implicit_variant", "rmsmp_last_device_status",
+)
+
+
+class rmsmp_layer(C.Structure):
+    _fields_ = [
+        ("magic", C.c_uint32),
+        ("M", C.c_int32), ("Cin", C.c_int32), ("kh", C.c_int32), ("kw", C.c_int32),
+        ("Cp", C.c_int32), ("Kp", C.c_int32),
+        ("nP", C.c_int32), ("nF4", C.c_int32), ("n8", C.c_int32),
+        ("nblocks", C.c_int32), ("reserved", C.c_int32),
+        ("off_perm", C.c_uint64), ("off_slot", C.c_uint64), ("off_wstep", C.c_uint64),
+        ("off_alpha", C.c_uint64), ("off_kind", C.c_uint64), ("off_blocks", C.c_uint64),
+        ("off_q4", C.c_uint64), ("off_q8", C.c_uint64),
+        ("packed_bytes", C.c_uint64),
+    ]
+
+    @property
+    def K(self) -> int:
+        return self.Cin * self.kh * self.kw
+
+
+class RmsmpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        try:
+            msg = lib().rmsmp_status_string(status).decode()
+        except Exception:
+            msg = "?"
+        super().__init__(f"{where}: status {status} ({msg})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the CUDA library; fails loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2111_00153_b200.build` "
+                "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.rmsmp_status_string.restype = C.c_char_p
+        L.rmsmp_status_string.argtypes = [C.c_int]
+        vp, i32, i64, f32 = C.c_void_p, C.c_int, C.c_int64, C.c_float
+        L.rmsmp_assign_rows.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp]
+        L.rmsmp_layer_init.argtypes = [C.POINTER(rmsmp_layer), i32, i32, i32, i32, vp, vp]
+        L.rmsmp_quantize_pack.argtypes = [vp, i32, C.POINTER(rmsmp_layer), vp, vp, vp, i32, vp,
+                                          C.c_size_t, vp]
+        L.rmsmp_unpack_codes.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, vp, vp]
+        L.rmsmp_quantize_act.argtypes = [vp, C.c_size_t, f32, i32, vp, C.POINTER(C.c_float), vp]
+        L.rmsmp_gemm.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
+        L.rmsmp_gemm_variant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i64, i64, f32, vp, i64,
+                                         i32, vp, i32, vp]
+        L.rmsmp_conv_implicit.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i32, i32, i32, i32, i32,
+                                          f32, vp, i32, vp, vp]
+        L.rmsmp_conv_implicit_variant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i32, i32, i32,
+                                                  i32, i32, f32, vp, i32, vp, i32, vp]
+        L.rmsmp_last_device_status.argtypes = [vp, vp]
+        _lib = L
+    return _lib
+
+
+def _dp(t):
+    """Device pointer of a torch tensor, or pass an int / None through."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return C.c_void_p(t)
+    return C.c_void_p(t.data_ptr())
+
+
+def _hp(a: np.ndarray):
+    return C.c_void_p(a.ctypes.data)
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return C.c_void_p(stream)
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _check(st: int, where: str):
+    if st != OK:
+        raise RmsmpError(st, where)
+
+
+def rmsmp_status_string(status: int) -> str:
+    return lib().rmsmp_status_string(status).decode()
+
+
+def rmsmp_assign_rows(h_W: np.ndarray, ratio):
+    """Host helper: (scheme, bits) uint8 arrays for ratio (PoT-4, Fixed-4, Fixed-8)."""
+    W = np.ascontiguousarray(h_W, dtype=np.float32)
+    W = W.reshape(W.shape[0], -1)
+    M, K = W.shape
+    scheme, bits = np.empty(M, np.uint8), np.empty(M, np.uint8)
+    _check(lib().rmsmp_assign_rows(_hp(W), M, K, int(ratio[0]), int(ratio[1]), int(ratio[2]),
+                                   _hp(scheme), _hp(bits)), "rmsmp_assign_rows")
+    return scheme, bits
+
+
+def rmsmp_layer_init(M: int, Cin: int, kh: int, kw: int, h_scheme, h_bits) -> rmsmp_layer:
+    scheme = np.ascontiguousarray(h_scheme, dtype=np.uint8)
+    bits = np.ascontiguousarray(h_bits, dtype=np.uint8)
+    if scheme.size != M or bits.size != M:
+        raise ValueError("scheme/bits need M entries")
+    layer = rmsmp_layer()
+    _check(lib().rmsmp_layer_init(C.byref(layer), M, Cin, kh, kw, _hp(scheme), _hp(bits)),
+           "rmsmp_layer_init")
+    return layer
+
+
+def rmsmp_quantize_pack(d_W, w_layout: int, layer: rmsmp_layer, h_scheme, h_bits, h_alpha,
+                        pot_mode: int, d_packed, packed_bytes: int | None = None, stream=None):
+    scheme = np.ascontiguousarray(h_scheme, dtype=np.uint8)
+    bits = np.ascontiguousarray(h_bits, dtype=np.uint8)
+    alpha = np.ascontiguousarray(h_alpha, dtype=np.float32)
+    if not (scheme.size == bits.size == alpha.size == layer.M):
+        raise ValueError("scheme/bits/alpha need M entries")
+    if packed_bytes is None:
+        packed_bytes = d_packed.numel() * d_packed.element_size()
+    _check(lib().rmsmp_quantize_pack(_dp(d_W), w_layout, C.byref(layer), _hp(scheme), _hp(bits),
+                                     _hp(alpha), pot_mode, _dp(d_packed), packed_bytes,
+                                     _stream(stream)), "rmsmp_quantize_pack")
+
+
+def rmsmp_unpack_codes(layer: rmsmp_layer, d_packed, d_values, d_perm=None, d_wstep=None,
+                       stream=None):
+    _check(lib().rmsmp_unpack_codes(C.byref(layer), _dp(d_packed), _dp(d_values), _dp(d_perm),
+                                    _dp(d_wstep), _stream(stream)), "rmsmp_unpack_codes")
+
+
+def rmsmp_quantize_act(d_X, count: int, alpha_a: float, kind: int, d_codes, stream=None) -> float:
+    """Returns the activation step (alpha_a/15 or alpha_a/7) as a Python float (fp32 value)."""
+    step = C.c_float(0.0)
+    _check(lib().rmsmp_quantize_act(_dp(d_X), count, alpha_a, kind, _dp(d_codes), C.byref(step),
+                                    _stream(stream)), "rmsmp_quantize_act")
+    return step.value
+
+
+def rmsmp_gemm(layer, d_packed, d_act, N: int, ld_act: int, act_step: float, d_out, ld_out: int,
+               out_layout: int = OUT_NM, d_acc=None, stream=None):
+    _check(lib().rmsmp_gemm(C.byref(layer), _dp(d_packed), _dp(d_act), N, ld_act, act_step,
+                            _dp(d_out), ld_out, out_layout, _dp(d_acc), _stream(stream)),
+           "rmsmp_gemm")
+
+
+def rmsmp_gemm_variant(layer, d_packed, d_act, N: int, ld_act: int, act_step: float, d_out,
+                       ld_out: int, out_layout: int, d_acc, variant: int, stream=None):
+    _check(lib().rmsmp_gemm_variant(C.byref(layer), _dp(d_packed), _dp(d_act), N, ld_act, act_step,
+                                    _dp(d_out), ld_out, out_layout, _dp(d_acc), variant,
+                                    _stream(stream)), "rmsmp_gemm_variant")
+
+
+def rmsmp_conv_implicit(layer, d_packed, d_act, B: int, H: int, W: int, stride: int, pad: int,
+                        act_step: float, d_out, out_layout: int = OUT_NM, d_acc=None, stream=None):
+    _check(lib().rmsmp_conv_implicit(C.byref(layer), _dp(d_packed), _dp(d_act), B, H, W, stride,
+                                     pad, act_step, _dp(d_out), out_layout, _dp(d_acc),
+                                     _stream(stream)), "rmsmp_conv_implicit")
+
+
+def rmsmp_conv_implicit_variant(layer, d_packed, d_act, B: int, H: int, W: int, stride: int,
+                                pad: int, act_step: float, d_out, out_layout: int, d_acc,
+                                variant: int, stream=None):
+    _check(lib().rmsmp_conv_implicit_variant(C.byref(layer), _dp(d_packed), _dp(d_act), B, H, W,
+                                             stride, pad, act_step, _dp(d_out), out_layout,
+                                             _dp(d_acc), variant, _stream(stream)),
+           "rmsmp_conv_implicit_variant")
+
+
+def rmsmp_last_device_status(d_packed, stream=None) -> int:
+    return lib().rmsmp_last_device_status(_dp(d_packed), _stream(stream))

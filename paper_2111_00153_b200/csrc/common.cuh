@@ -1,0 +1,89 @@
+// Internal declarations shared by the translation units of librmsmp (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "../../include/rmsmp.h"
+
+namespace rmsmp {
+
+constexpr uint32_t kLayerMagic = 0x524D5350u;   // "RMSP"
+constexpr uint32_t kBlobVersion = 1u;
+constexpr int kBlockRows = 128;                  // rows of one MMA tile = one entry of `blocks`
+constexpr int kStatusOffset = 64;                // byte offset of the device status word
+
+enum RowKind : int { kPoT4 = 0, kFixed4 = 1, kFixed8 = 2 };
+
+// First 256 bytes of a packed buffer.
+struct BlobHeader {
+    uint32_t magic, version;
+    int32_t M, Cin, kh, kw, Cp, Kp, nP, nF4, n8, nblocks, pot_mode;
+    int32_t pad0[3];
+    uint32_t status;          // byte 64
+    uint32_t pad1[47];
+};
+static_assert(sizeof(BlobHeader) == 256, "header is 256 bytes");
+static_assert(offsetof(BlobHeader, status) == kStatusOffset, "status word at byte 64");
+
+// Everything a contraction kernel needs; passed by value.
+struct Problem {
+    // weights
+    const uint8_t* blob;
+    const int32_t* perm;      // packed position -> original row
+    const int32_t* slot;      // original row -> packed position
+    const float* wstep;       // by original row
+    const uint8_t* kind;      // by original row
+    const int32_t* blocks;    // [nblocks][8]
+    const uint8_t* q4;        // [(nP+nF4)][Kp/2]
+    const uint8_t* q8;        // [n8][Kp]
+    uint32_t* status;
+    int M, Cin, kh, kw, Cp, Kp, nP, nF4, n8, nblocks;
+    // activations: [B][H][W] pixels of `pix_pitch` bytes, Cin codes used in each
+    const int8_t* act;
+    int B, H, W, Ho, Wo, stride, pad;
+    int64_t pix_pitch;
+    int64_t N;                // B*Ho*Wo
+    // outputs
+    float act_step;
+    float* out;
+    int32_t* acc;             // may be null
+    int64_t ld_out;
+    int out_mn;               // 0: y[n*ld+m], 1: y[m*ld+n]
+};
+
+// kernels (each returns the CUDA launch error, cudaSuccess if fine)
+cudaError_t launch_pack(const float* dW, int conv_oihw, const rmsmp_layer& L, int pot_mode,
+                        uint8_t* blob, cudaStream_t st);
+cudaError_t launch_unpack(const rmsmp_layer& L, const uint8_t* blob, int8_t* values,
+                          int32_t* perm, float* wstep, cudaStream_t st);
+cudaError_t launch_quantize_act(const float* x, size_t count, float alpha, int kind, int8_t* codes,
+                                cudaStream_t st);
+cudaError_t launch_simple(const Problem& p, cudaStream_t st);
+cudaError_t launch_simt(const Problem& p, bool shiftadd, cudaStream_t st);
+// returns false if the tensor variant cannot run this problem (alignment / shape)
+bool tensor_supported(const Problem& p);
+rmsmp_status launch_tensor(const Problem& p, cudaStream_t st);
+
+// ---- device helpers used by more than one kernel file ----
+
+// Integer value of a PoT-4 nibble (sign<<3 | e): 0 or +-2^(e-1).
+__device__ __forceinline__ int pot_value(int nib)
+{
+    int e = nib & 7;
+    int v = e ? (1 << (e - 1)) : 0;
+    return (nib & 8) ? -v : v;
+}
+
+// Value of code k' of packed row `row4` (4-bit storage), see the layout in rmsmp.h.
+__device__ __forceinline__ int decode4(const uint8_t* row4, int kprime, int kind)
+{
+    int chunk = kprime >> 5, o = kprime & 31;
+    if (kind == kPoT4) {
+        int byte = row4[chunk * 16 + (o >> 1)];
+        return pot_value((o & 1) ? (byte >> 4) : (byte & 15));
+    }
+    int byte = row4[chunk * 16 + (o & 15)];
+    int nib = (o < 16) ? (byte >> 4) : (byte & 15);
+    return (nib ^ 8) - 8;
+}
+
+}  // namespace rmsmp

@@ -1,0 +1,362 @@
+// Host side of the C ABI: validation, layer description, metadata upload, dispatch.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <vector>
+#include "common.cuh"
+
+using namespace rmsmp;
+
+namespace {
+
+inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+inline int row_kind(int scheme, int bits)
+{
+    if (scheme == RMSMP_SCHEME_POT && bits == 4) return kPoT4;
+    if (scheme == RMSMP_SCHEME_FIXED && bits == 4) return kFixed4;
+    if (scheme == RMSMP_SCHEME_FIXED && bits == 8) return kFixed8;
+    return -1;
+}
+
+bool layer_ok(const rmsmp_layer* L)
+{
+    return L && L->magic == kLayerMagic && L->M >= 1 && L->Cin >= 1 && L->kh >= 1 && L->kw >= 1 &&
+           L->nP + L->nF4 + L->n8 == L->M && L->packed_bytes >= 256;
+}
+
+rmsmp_status check_arch()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return RMSMP_ERR_CUDA; }
+    static int cached_major[64];
+    static bool have[64];
+    if (dev < 0 || dev >= 64) return RMSMP_ERR_CUDA;
+    if (!have[dev]) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return RMSMP_ERR_CUDA;
+        }
+        cached_major[dev] = major;
+        have[dev] = true;
+    }
+    return cached_major[dev] == 10 ? RMSMP_OK : RMSMP_ERR_ARCH;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+void fill_problem(Problem& p, const rmsmp_layer* L, const void* d_packed)
+{
+    const uint8_t* blob = static_cast<const uint8_t*>(d_packed);
+    p.blob = blob;
+    p.perm = reinterpret_cast<const int32_t*>(blob + L->off_perm);
+    p.slot = reinterpret_cast<const int32_t*>(blob + L->off_slot);
+    p.wstep = reinterpret_cast<const float*>(blob + L->off_wstep);
+    p.kind = blob + L->off_kind;
+    p.blocks = reinterpret_cast<const int32_t*>(blob + L->off_blocks);
+    p.q4 = blob + L->off_q4;
+    p.q8 = blob + L->off_q8;
+    p.status = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(blob) + kStatusOffset);
+    p.M = L->M; p.Cin = L->Cin; p.kh = L->kh; p.kw = L->kw; p.Cp = L->Cp; p.Kp = L->Kp;
+    p.nP = L->nP; p.nF4 = L->nF4; p.n8 = L->n8; p.nblocks = L->nblocks;
+}
+
+rmsmp_status dispatch(Problem& p, rmsmp_variant variant, cudaStream_t st)
+{
+    if (variant == RMSMP_VARIANT_AUTO) {
+        if (p.N >= 32 && tensor_supported(p)) variant = RMSMP_VARIANT_TENSOR;
+        else variant = RMSMP_VARIANT_SIMT;
+    }
+    cudaError_t e = cudaSuccess;
+    switch (variant) {
+        case RMSMP_VARIANT_TENSOR:
+            if (!tensor_supported(p)) return RMSMP_ERR_VARIANT;
+            return launch_tensor(p, st);
+        case RMSMP_VARIANT_SIMT: e = launch_simt(p, false, st); break;
+        case RMSMP_VARIANT_SHIFTADD: e = launch_simt(p, true, st); break;
+        case RMSMP_VARIANT_SIMPLE: e = launch_simple(p, st); break;
+        default: return RMSMP_ERR_VARIANT;
+    }
+    return e == cudaSuccess ? RMSMP_OK : RMSMP_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rmsmp_status_string(rmsmp_status s)
+{
+    switch (s) {
+        case RMSMP_OK: return "ok";
+        case RMSMP_ERR_NULL: return "null pointer";
+        case RMSMP_ERR_SHAPE: return "bad shape";
+        case RMSMP_ERR_SCHEME: return "scheme/bits not in {PoT-4, Fixed-4, Fixed-8}";
+        case RMSMP_ERR_SCALE: return "clip value not finite and positive";
+        case RMSMP_ERR_ALIGN: return "pointer or leading dimension not 16-byte aligned";
+        case RMSMP_ERR_BUFFER_TOO_SMALL: return "packed buffer too small";
+        case RMSMP_ERR_ARCH: return "device is not sm_100";
+        case RMSMP_ERR_CUDA: return "CUDA call failed";
+        case RMSMP_ERR_TIMEOUT: return "bounded device wait ran out";
+        case RMSMP_ERR_BAD_LAYER: return "layer descriptor not initialised";
+        case RMSMP_ERR_VARIANT: return "kernel variant cannot run this problem";
+    }
+    return "unknown status";
+}
+
+rmsmp_status rmsmp_assign_rows(const float* h_W, int M, int K, int A, int B, int C,
+                               uint8_t* h_scheme, uint8_t* h_bits)
+{
+    if (!h_W || !h_scheme || !h_bits) return RMSMP_ERR_NULL;
+    if (M < 1 || K < 1 || A < 0 || B < 0 || C < 0 || A + B + C != 100) return RMSMP_ERR_SHAPE;
+    // population variance per row, double, two plain passes
+    std::vector<std::pair<double, int>> rank((size_t)M);
+    for (int r = 0; r < M; ++r) {
+        const float* w = h_W + (size_t)r * K;
+        double sum = 0.0;
+        for (int k = 0; k < K; ++k) sum += (double)w[k];
+        const double mean = sum / (double)K;
+        double ss = 0.0;
+        for (int k = 0; k < K; ++k) {
+            const double d = (double)w[k] - mean;
+            ss += d * d;
+        }
+        rank[(size_t)r] = {ss / (double)K, r};
+    }
+    std::sort(rank.begin(), rank.end());   // (variance, row) ascending
+    int n8 = (int)std::floor((double)M * C / 100.0 + 0.5);
+    n8 = std::min(n8, M);
+    int nP = (int)std::floor((double)M * A / 100.0 + 0.5);
+    nP = std::min(nP, M - n8);
+    for (int i = 0; i < M; ++i) {
+        const int r = rank[(size_t)i].second;
+        if (i < nP) { h_scheme[r] = RMSMP_SCHEME_POT; h_bits[r] = 4; }
+        else if (i < M - n8) { h_scheme[r] = RMSMP_SCHEME_FIXED; h_bits[r] = 4; }
+        else { h_scheme[r] = RMSMP_SCHEME_FIXED; h_bits[r] = 8; }
+    }
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_layer_init(rmsmp_layer* L, int M, int Cin, int kh, int kw,
+                              const uint8_t* h_scheme, const uint8_t* h_bits)
+{
+    if (!L || !h_scheme || !h_bits) return RMSMP_ERR_NULL;
+    if (M < 1 || M > (1 << 20) || Cin < 1 || kh < 1 || kw < 1 || kh > 16 || kw > 16)
+        return RMSMP_ERR_SHAPE;
+    if ((int64_t)Cin * kh * kw > 1000000) return RMSMP_ERR_SHAPE;
+    int cnt[3] = {0, 0, 0};
+    for (int r = 0; r < M; ++r) {
+        const int k = row_kind(h_scheme[r], h_bits[r]);
+        if (k < 0) return RMSMP_ERR_SCHEME;
+        ++cnt[k];
+    }
+    std::memset(L, 0, sizeof(*L));
+    L->magic = kLayerMagic;
+    L->M = M; L->Cin = Cin; L->kh = kh; L->kw = kw;
+    L->Cp = (Cin + 31) / 32 * 32;
+    L->Kp = (int32_t)align_up((uint64_t)kh * kw * L->Cp, 128);
+    if (kh * kw > 1 && L->Kp > 196608) return RMSMP_ERR_SHAPE;   // one shared-memory segment in the pack kernel
+    L->nP = cnt[0]; L->nF4 = cnt[1]; L->n8 = cnt[2];
+    L->nblocks = (M + kBlockRows - 1) / kBlockRows;
+    uint64_t off = 256;
+    L->off_perm = off;   off = align_up(off + 4ull * M, 256);
+    L->off_slot = off;   off = align_up(off + 4ull * M, 256);
+    L->off_wstep = off;  off = align_up(off + 4ull * M, 256);
+    L->off_alpha = off;  off = align_up(off + 4ull * M, 256);
+    L->off_kind = off;   off = align_up(off + 1ull * M, 256);
+    L->off_blocks = off; off = align_up(off + 32ull * L->nblocks, 256);
+    L->off_q4 = off;     off = align_up(off + (uint64_t)(cnt[0] + cnt[1]) * (L->Kp / 2), 256);
+    L->off_q8 = off;     off = align_up(off + (uint64_t)cnt[2] * L->Kp, 256);
+    L->packed_bytes = off;
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_quantize_pack(const float* d_W, rmsmp_w_layout w_layout, const rmsmp_layer* L,
+                                 const uint8_t* h_scheme, const uint8_t* h_bits,
+                                 const float* h_alpha, rmsmp_pot_mode pot_mode, void* d_packed,
+                                 size_t packed_bytes, void* stream)
+{
+    if (!d_W || !L || !h_scheme || !h_bits || !h_alpha || !d_packed) return RMSMP_ERR_NULL;
+    if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+    if (w_layout != RMSMP_W_LINEAR && w_layout != RMSMP_W_CONV_OIHW) return RMSMP_ERR_SHAPE;
+    if (w_layout == RMSMP_W_LINEAR && (L->kh != 1 || L->kw != 1)) return RMSMP_ERR_SHAPE;
+    if (pot_mode != RMSMP_POT_NEAREST && pot_mode != RMSMP_POT_LOG2) return RMSMP_ERR_SCHEME;
+    if (packed_bytes < L->packed_bytes) return RMSMP_ERR_BUFFER_TOO_SMALL;
+    if (!aligned16(d_W) || (reinterpret_cast<uintptr_t>(d_packed) & 255) != 0) return RMSMP_ERR_ALIGN;
+    const int M = L->M;
+    int cnt[3] = {0, 0, 0};
+    for (int r = 0; r < M; ++r) {
+        const int k = row_kind(h_scheme[r], h_bits[r]);
+        if (k < 0) return RMSMP_ERR_SCHEME;
+        ++cnt[k];
+        if (!(h_alpha[r] > 0.0f) || !std::isfinite(h_alpha[r])) return RMSMP_ERR_SCALE;
+    }
+    if (cnt[0] != L->nP || cnt[1] != L->nF4 || cnt[2] != L->n8) return RMSMP_ERR_SCHEME;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+
+    // metadata: everything before the code regions, built on the host and sent in one copy
+    std::vector<uint8_t> meta((size_t)L->off_q4, 0);
+    BlobHeader* H = reinterpret_cast<BlobHeader*>(meta.data());
+    H->magic = kLayerMagic; H->version = kBlobVersion;
+    H->M = M; H->Cin = L->Cin; H->kh = L->kh; H->kw = L->kw; H->Cp = L->Cp; H->Kp = L->Kp;
+    H->nP = L->nP; H->nF4 = L->nF4; H->n8 = L->n8; H->nblocks = L->nblocks; H->pot_mode = pot_mode;
+    H->status = 0;
+    int32_t* perm = reinterpret_cast<int32_t*>(meta.data() + L->off_perm);
+    int32_t* slot = reinterpret_cast<int32_t*>(meta.data() + L->off_slot);
+    float* wstep = reinterpret_cast<float*>(meta.data() + L->off_wstep);
+    float* alpha = reinterpret_cast<float*>(meta.data() + L->off_alpha);
+    uint8_t* kind = meta.data() + L->off_kind;
+    int32_t* blocks = reinterpret_cast<int32_t*>(meta.data() + L->off_blocks);
+    int next[3] = {0, cnt[0], cnt[0] + cnt[1]};          // stable grouping
+    for (int r = 0; r < M; ++r) {
+        const int k = row_kind(h_scheme[r], h_bits[r]);
+        const int blk = r / kBlockRows;
+        int32_t* be = blocks + 8 * blk;
+        const int rel = next[k] - (k == 0 ? 0 : (k == 1 ? cnt[0] : cnt[0] + cnt[1]));
+        if (be[2 * k + 1] == 0) be[2 * k] = rel;
+        be[2 * k + 1] += 1;
+        perm[next[k]] = r;
+        slot[r] = next[k];
+        ++next[k];
+        kind[r] = (uint8_t)k;
+        alpha[r] = h_alpha[r];
+        const float q = (k == kPoT4) ? 64.0f : (k == kFixed4 ? 7.0f : 127.0f);
+        wstep[r] = h_alpha[r] / q;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(d_packed, meta.data(), meta.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    if (launch_pack(d_W, w_layout == RMSMP_W_CONV_OIHW, *L, pot_mode, static_cast<uint8_t*>(d_packed), st) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_unpack_codes(const rmsmp_layer* L, const void* d_packed, int8_t* d_values,
+                                int32_t* d_perm, float* d_wstep, void* stream)
+{
+    if (!L || !d_packed || !d_values) return RMSMP_ERR_NULL;
+    if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    if (launch_unpack(*L, static_cast<const uint8_t*>(d_packed), d_values, d_perm, d_wstep,
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_quantize_act(const float* d_X, size_t count, float alpha_a, rmsmp_act_kind kind,
+                                int8_t* d_codes, float* h_act_step, void* stream)
+{
+    if (!d_X || !d_codes) return RMSMP_ERR_NULL;
+    if (count < 1) return RMSMP_ERR_SHAPE;
+    if (kind != RMSMP_ACT_U4 && kind != RMSMP_ACT_S4) return RMSMP_ERR_SCHEME;
+    if (!(alpha_a > 0.0f) || !std::isfinite(alpha_a)) return RMSMP_ERR_SCALE;
+    if (h_act_step) *h_act_step = alpha_a / (kind == RMSMP_ACT_U4 ? 15.0f : 7.0f);
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    if (launch_quantize_act(d_X, count, alpha_a, kind, d_codes, static_cast<cudaStream_t>(stream)) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_gemm_variant(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act,
+                                int64_t N, int64_t ld_act, float act_step, float* d_out,
+                                int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
+                                rmsmp_variant variant, void* stream)
+{
+    if (!L || !d_packed || !d_act || !d_out) return RMSMP_ERR_NULL;
+    if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+    if (L->kh != 1 || L->kw != 1) return RMSMP_ERR_SHAPE;
+    if (N < 1 || N > (int64_t)1 << 31 || ld_act < L->Cin) return RMSMP_ERR_SHAPE;
+    if (out_layout != RMSMP_OUT_NM && out_layout != RMSMP_OUT_MN) return RMSMP_ERR_SHAPE;
+    if (ld_out < (out_layout == RMSMP_OUT_NM ? (int64_t)L->M : N)) return RMSMP_ERR_SHAPE;
+    if (!std::isfinite(act_step)) return RMSMP_ERR_SCALE;
+    if (!aligned16(d_act) || !aligned16(d_out) || (d_acc && !aligned16(d_acc)) || (ld_act & 15) ||
+        (reinterpret_cast<uintptr_t>(d_packed) & 255))
+        return RMSMP_ERR_ALIGN;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    Problem p;
+    fill_problem(p, L, d_packed);
+    p.act = d_act;
+    p.B = (int)std::min<int64_t>(N, 0x7fffffff); p.H = 1; p.W = 1; p.Ho = 1; p.Wo = 1; p.stride = 1; p.pad = 0;
+    p.pix_pitch = ld_act; p.N = N;
+    p.act_step = act_step; p.out = d_out; p.acc = d_acc; p.ld_out = ld_out;
+    p.out_mn = (out_layout == RMSMP_OUT_MN);
+    return dispatch(p, variant, static_cast<cudaStream_t>(stream));
+}
+
+rmsmp_status rmsmp_gemm(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act, int64_t N,
+                        int64_t ld_act, float act_step, float* d_out, int64_t ld_out,
+                        rmsmp_out_layout out_layout, int32_t* d_acc, void* stream)
+{
+    return rmsmp_gemm_variant(L, d_packed, d_act, N, ld_act, act_step, d_out, ld_out, out_layout,
+                              d_acc, RMSMP_VARIANT_AUTO, stream);
+}
+
+rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* L, const void* d_packed,
+                                         const int8_t* d_act, int B, int H, int W, int stride,
+                                         int pad, float act_step, float* d_out,
+                                         rmsmp_out_layout out_layout, int32_t* d_acc,
+                                         rmsmp_variant variant, void* stream)
+{
+    if (!L || !d_packed || !d_act || !d_out) return RMSMP_ERR_NULL;
+    if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+    if (B < 1 || H < 1 || W < 1 || stride < 1 || stride > 8 || pad < 0 || pad > 16) return RMSMP_ERR_SHAPE;
+    if (H + 2 * pad < L->kh || W + 2 * pad < L->kw) return RMSMP_ERR_SHAPE;
+    if (out_layout != RMSMP_OUT_NM && out_layout != RMSMP_OUT_MN) return RMSMP_ERR_SHAPE;
+    if (!std::isfinite(act_step)) return RMSMP_ERR_SCALE;
+    const int Ho = (H + 2 * pad - L->kh) / stride + 1, Wo = (W + 2 * pad - L->kw) / stride + 1;
+    const int64_t N = (int64_t)B * Ho * Wo;
+    if (N > (int64_t)1 << 31 || (int64_t)B * H * W > (int64_t)1 << 31) return RMSMP_ERR_SHAPE;
+    if (!aligned16(d_act) || !aligned16(d_out) || (d_acc && !aligned16(d_acc)) ||
+        (reinterpret_cast<uintptr_t>(d_packed) & 255))
+        return RMSMP_ERR_ALIGN;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    Problem p;
+    fill_problem(p, L, d_packed);
+    p.act = d_act;
+    p.B = B; p.H = H; p.W = W; p.Ho = Ho; p.Wo = Wo; p.stride = stride; p.pad = pad;
+    p.pix_pitch = L->Cin; p.N = N;
+    p.act_step = act_step; p.out = d_out; p.acc = d_acc;
+    p.out_mn = (out_layout == RMSMP_OUT_MN);
+    p.ld_out = p.out_mn ? N : L->M;
+    return dispatch(p, variant, static_cast<cudaStream_t>(stream));
+}
+
+rmsmp_status rmsmp_conv_implicit(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act,
+                                 int B, int H, int W, int stride, int pad, float act_step,
+                                 float* d_out, rmsmp_out_layout out_layout, int32_t* d_acc,
+                                 void* stream)
+{
+    return rmsmp_conv_implicit_variant(L, d_packed, d_act, B, H, W, stride, pad, act_step, d_out,
+                                       out_layout, d_acc, RMSMP_VARIANT_AUTO, stream);
+}
+
+rmsmp_status rmsmp_last_device_status(const void* d_packed, void* stream)
+{
+    if (!d_packed) return RMSMP_ERR_NULL;
+    uint32_t w = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&w, static_cast<const uint8_t*>(d_packed) + kStatusOffset, 4,
+                        cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return w <= RMSMP_ERR_VARIANT ? (rmsmp_status)w : RMSMP_ERR_CUDA;
+}
+
+}  // extern "C"

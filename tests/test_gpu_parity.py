@@ -1,0 +1,257 @@
+"""GPU parity: every step of the CUDA path against the CPU oracle, through the C ABI.
+
+Integer results (codes, permutation, accumulators) must match bit for bit; fp32 outputs are a
+single multiply of exactly converted integers and must match bit for bit too, and lie within
+1e-6 relative of the double-precision value.
+"""
+import numpy as np
+import pytest
+
+from oracle import rmsmp_oracle as O
+from paper_2111_00153_b200 import binding as R
+from paper_2111_00153_b200 import synth
+from tests import harness as Hn
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = [R.VARIANT_SIMPLE, R.VARIANT_SIMT, R.VARIANT_SHIFTADD, R.VARIANT_TENSOR]
+VNAME = {R.VARIANT_SIMPLE: "simple", R.VARIANT_SIMT: "simt", R.VARIANT_SHIFTADD: "shiftadd",
+         R.VARIANT_TENSOR: "tensor", R.VARIANT_AUTO: "auto"}
+
+
+def _mixed_map(M, seed, ratio=(60, 35, 5)):
+    """A scheme map with the given ratio, rows shuffled (independent of weight values)."""
+    nP, nF4, n8 = O.ratio_counts(M, ratio)
+    kinds = np.array([0] * nP + [1] * nF4 + [2] * n8)
+    np.random.default_rng(seed).shuffle(kinds)
+    scheme = np.where(kinds == 0, 0, 1).astype(np.uint8)
+    bits = np.where(kinds == 2, 8, 4).astype(np.uint8)
+    return scheme, bits
+
+
+def _check_layer_outputs(y, acc, acc_ref, ws, act_step, alpha, scheme, bits):
+    assert np.array_equal(acc, acc_ref)
+    y_ref = O.epilogue(acc_ref, ws, act_step)
+    assert np.array_equal(y.view(np.uint32), y_ref.view(np.uint32))
+    Qw = np.where(scheme == 0, 64.0, np.where(bits == 4, 7.0, 127.0))
+    dbl = acc_ref.astype(np.float64) * (alpha.astype(np.float64) / Qw)[None, :] * float(act_step)
+    nz = dbl != 0
+    assert np.all(np.abs(y[nz] - dbl[nz]) <= 1e-6 * np.abs(dbl[nz]))
+
+
+# ------------------------------------------------------------------ pack / unpack
+
+@pytest.mark.parametrize("M,K,ratio", [(256, 512, (60, 35, 5)), (37, 200, (50, 40, 10)),
+                                       (5, 3, (0, 100, 0)), (130, 1000, (100, 0, 0)),
+                                       (64, 40000, (60, 35, 5)), (3, 7, (34, 33, 33))])
+@pytest.mark.parametrize("mode", [R.POT_NEAREST, R.POT_LOG2])
+def test_pack_codes_linear(M, K, ratio, mode):
+    if mode == R.POT_LOG2 and K > 2000:
+        pytest.skip("one large case per mode is enough")
+    W = synth.weights_normal(synth.rng(70, M + K), (M, K))
+    W[0, :min(K, 8)] = [0, 1e-9, -1e-9, 1, -1, 0.02, -0.02, 3e-4][:min(K, 8)]
+    scheme, bits = O.assign_rows(W, ratio)
+    alpha = synth.alpha_rows(W)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha, mode)
+    vals, perm, ws = Hn.unpack(layer, d_packed)
+    v_ref, ws_ref = O.quantize_rows(W, scheme, bits, alpha, mode)
+    assert np.array_equal(vals, v_ref)
+    assert np.array_equal(perm, O.group_rows(scheme, bits))
+    assert np.array_equal(ws.view(np.uint32), ws_ref.view(np.uint32))
+
+
+def test_pack_codes_on_rounding_ties_and_midpoints():
+    # weights placed exactly on Fixed rounding ties and PoT decision points, alpha = 1
+    ties4 = [np.float32((j + 0.5) / 7.0) for j in range(7)]
+    ties8 = [np.float32((j + 0.5) / 127.0) for j in range(0, 127, 9)]
+    mids = [2.0 ** -7] + [3 * 2.0 ** (k - 9) for k in range(2, 8)]
+    geo = [2.0 ** -(j + 0.5) for j in range(7)]
+    pts = []
+    for v in ties4 + ties8 + mids + geo:
+        f = np.float32(v)
+        pts += [f, np.nextafter(f, np.float32(0)), np.nextafter(f, np.float32(2)), -f]
+    K = len(pts)
+    W = np.tile(np.array(pts, np.float32), (6, 1))
+    scheme = np.array([0, 1, 1, 0, 1, 1], np.uint8)
+    bits = np.array([4, 4, 8, 4, 4, 8], np.uint8)
+    alpha = np.array([1, 1, 1, 0.5, 0.5, 0.5], np.float32)
+    for mode in (R.POT_NEAREST, R.POT_LOG2):
+        layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha, mode)
+        vals, _, _ = Hn.unpack(layer, d_packed)
+        v_ref, _ = O.quantize_rows(W, scheme, bits, alpha, mode)
+        assert np.array_equal(vals, v_ref)
+
+
+@pytest.mark.parametrize("M,Cin,k", [(64, 64, 3), (20, 24, 3), (9, 5, 1), (12, 40, 5), (130, 16, 2)])
+def test_pack_codes_conv(M, Cin, k):
+    W = synth.weights_kaiming(synth.rng(71, M + Cin), M, Cin, k, k)
+    scheme, bits = O.assign_rows(W, (60, 35, 5))
+    alpha = synth.alpha_rows(W)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    vals, perm, ws = Hn.unpack(layer, d_packed)
+    v_ref, ws_ref = O.quantize_rows(W.reshape(M, -1), scheme, bits, alpha)
+    assert np.array_equal(vals, v_ref)
+    assert np.array_equal(perm, O.group_rows(scheme, bits))
+
+
+# ------------------------------------------------------------------ activation quantizer
+
+@pytest.mark.parametrize("count", [1, 15, 16, 1000, 4099, 1 << 20])
+@pytest.mark.parametrize("kind", [R.ACT_U4, R.ACT_S4])
+def test_quantize_act(count, kind):
+    g = synth.rng(72, count)
+    x = synth.act_halfnormal(g, count) if kind == R.ACT_U4 else synth.act_normal(g, count)
+    x[: min(count, 6)] = [0.0, 0.1, 0.3, 3.0, 1.5, 2.9999][: min(count, 6)]
+    codes, step = Hn.quantize_act(x, synth.ALPHA_ACT, kind)
+    c_ref, s_ref = O.quantize_act(x, synth.ALPHA_ACT, kind)
+    assert np.array_equal(codes, c_ref)
+    assert step == s_ref
+
+
+# ------------------------------------------------------------------ linear layer
+
+LIN_CASES = [
+    # M, K, N, ratio        spans several 128-row blocks / 256-token tiles with ragged tails
+    (256, 512, 64, (60, 35, 5)),        # config 1
+    (128, 128, 256, (60, 35, 5)),
+    (300, 200, 77, (50, 40, 10)),
+    (130, 96, 513, (60, 35, 5)),
+    (64, 576, 300, (65, 30, 5)),
+    (1, 32, 1, (0, 100, 0)),
+    (200, 48, 40, (0, 0, 100)),
+    (150, 1000, 33, (100, 0, 0)),
+    (257, 2304, 260, (60, 35, 5)),
+]
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=lambda v: VNAME[v])
+@pytest.mark.parametrize("M,K,N,ratio", LIN_CASES)
+def test_linear_layer(M, K, N, ratio, variant):
+    g = synth.rng(73, M * 7 + K + N)
+    W = synth.weights_normal(g, (M, K))
+    scheme, bits = _mixed_map(M, M + K, ratio)
+    alpha = synth.alpha_rows(W)
+    signed = (M % 2 == 0)
+    act = g.integers(-7, 8, (N, K), dtype=np.int8) if signed else synth.act_codes_uniform(g, (N, K))
+    act_step = np.float32(0.1)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    try:
+        y, acc = Hn.gemm(layer, d_packed, act, act_step, variant)
+    except R.RmsmpError as e:
+        if e.status == R.ERR_VARIANT and variant == R.VARIANT_TENSOR and K % 16 != 0:
+            pytest.skip("tensor variant needs K % 16 == 0")
+        raise
+    v_ref, ws = O.quantize_rows(W, scheme, bits, alpha)
+    acc_ref = O.matmul(v_ref, act)
+    _check_layer_outputs(y, acc, acc_ref, ws, act_step, alpha, scheme, bits)
+
+
+@pytest.mark.parametrize("variant", [R.VARIANT_SIMT, R.VARIANT_TENSOR, R.VARIANT_AUTO], ids=lambda v: VNAME[v])
+def test_linear_layer_mn_layout_and_padded_ld(variant):
+    M, K, N = 140, 160, 70
+    g = synth.rng(74, variant)
+    W = synth.weights_normal(g, (M, K))
+    scheme, bits = O.assign_rows(W, (60, 35, 5))
+    alpha = synth.alpha_rows(W)
+    act = synth.act_codes_uniform(g, (N, K))
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    y, acc = Hn.gemm(layer, d_packed, act, 0.25, variant, out_layout=R.OUT_MN, ld_act=192)
+    v_ref, ws = O.quantize_rows(W, scheme, bits, alpha)
+    _check_layer_outputs(y, acc, O.matmul(v_ref, act), ws, np.float32(0.25), alpha, scheme, bits)
+    y2, _ = Hn.gemm(layer, d_packed, act, 0.25, variant, want_acc=False)
+    assert np.array_equal(y2, y)
+
+
+def test_extreme_codes_do_not_overflow_or_lose_bits():
+    # every weight at full scale, every activation at 15: |acc| = K*127*15 on Fixed-8 rows
+    M, K, N = 130, 4608, 40
+    W = np.ones((M, K), np.float32)
+    W[::2] = -1
+    scheme, bits = _mixed_map(M, 5, (40, 30, 30))
+    alpha = np.ones(M, np.float32)
+    act = np.full((N, K), 15, np.int8)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    v_ref, ws = O.quantize_rows(W, scheme, bits, alpha)
+    acc_ref = O.matmul(v_ref, act)
+    assert np.array_equal(acc_ref.astype(np.int64), O.matmul_i64(v_ref, act))
+    assert np.abs(acc_ref).max() == K * 127 * 15
+    for variant in VARIANTS:
+        y, acc = Hn.gemm(layer, d_packed, act, 1.0, variant)
+        _check_layer_outputs(y, acc, acc_ref, ws, np.float32(1.0), alpha, scheme, bits)
+
+
+# ------------------------------------------------------------------ convolution
+
+CONV_CASES = [
+    # M, Cin, k, stride, pad, B, H, W
+    (64, 64, 3, 1, 1, 2, 14, 14),
+    (40, 32, 3, 2, 1, 3, 14, 14),
+    (130, 128, 3, 1, 1, 2, 7, 7),
+    (24, 16, 1, 2, 0, 2, 8, 8),
+    (16, 16, 1, 1, 0, 1, 5, 9),
+    (32, 48, 3, 2, 1, 2, 9, 12),      # odd sizes, non-square
+    (140, 256, 3, 1, 1, 5, 7, 7),     # several images per tile, ragged last tile
+    (20, 20, 3, 1, 1, 1, 6, 6),       # Cin not a multiple of 16: CUDA-core variants only
+    (64, 64, 3, 1, 1, 1, 56, 56),
+]
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=lambda v: VNAME[v])
+@pytest.mark.parametrize("M,Cin,k,stride,pad,B,H,W", CONV_CASES)
+def test_conv_layer(M, Cin, k, stride, pad, B, H, W, variant):
+    g = synth.rng(75, M + Cin + H)
+    Wt = synth.weights_kaiming(g, M, Cin, k, k)
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    alpha = synth.alpha_rows(Wt)
+    x = synth.act_halfnormal(g, (B, H, W, Cin))
+    codes, act_step = O.quantize_act(x, synth.ALPHA_ACT, O.ACT_U4)
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    try:
+        y, acc = Hn.conv(layer, d_packed, codes, stride, pad, act_step, variant)
+    except R.RmsmpError as e:
+        if e.status == R.ERR_VARIANT and variant == R.VARIANT_TENSOR and Cin % 16 != 0:
+            pytest.skip("tensor variant needs Cin % 16 == 0")
+        raise
+    v_ref, ws, acc_ref, y_ref = O.layer_conv(Wt, scheme, bits, alpha, codes, act_step, stride, pad)
+    acc_ref = acc_ref.reshape(-1, M)
+    _check_layer_outputs(y, acc, acc_ref, ws, act_step, alpha, scheme, bits)
+
+
+def test_conv_mn_layout_auto():
+    M, Cin, B, H = 72, 32, 2, 10
+    g = synth.rng(76)
+    Wt = synth.weights_kaiming(g, M, Cin, 3, 3)
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    alpha = synth.alpha_rows(Wt)
+    codes = synth.act_codes_uniform(g, (B, H, H, Cin))
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    y, acc = Hn.conv(layer, d_packed, codes, 1, 1, 0.2, R.VARIANT_AUTO, out_layout=R.OUT_MN)
+    _, ws, acc_ref, _ = O.layer_conv(Wt, scheme, bits, alpha, codes, np.float32(0.2), 1, 1)
+    _check_layer_outputs(y, acc, acc_ref.reshape(-1, M), ws, np.float32(0.2), alpha, scheme, bits)
+
+
+# ------------------------------------------------------------------ the whole path, one call after the other
+
+def test_full_path_fp32_in_fp32_out():
+    """quantize_pack -> quantize_act -> conv, from fp32 tensors, as the benchmark runs it."""
+    import torch
+    L = synth.ConvShape("t", 96, 64, 3, 1, 1, 14)
+    g = synth.rng(77)
+    Wt = synth.weights_kaiming(g, L.M, L.Cin, 3, 3)
+    x = synth.act_halfnormal(g, (4, 14, 14, 64))
+    scheme, bits = R.rmsmp_assign_rows(Wt, synth.RATIO_RMSMP1)
+    s2, b2 = O.assign_rows(Wt, synth.RATIO_RMSMP1)
+    assert np.array_equal(scheme, s2) and np.array_equal(bits, b2)
+    alpha = synth.alpha_rows(Wt)
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    dx = torch.from_numpy(x).cuda()
+    dc = torch.empty(x.shape, dtype=torch.int8, device="cuda")
+    step = R.rmsmp_quantize_act(dx, dx.numel(), synth.ALPHA_ACT, R.ACT_U4, dc)
+    N = 4 * 14 * 14
+    y = torch.empty((N, L.M), dtype=torch.float32, device="cuda")
+    R.rmsmp_conv_implicit(layer, d_packed, dc, 4, 14, 14, 1, 1, step, y)
+    torch.cuda.synchronize()
+    codes, st_ref = O.quantize_act(x, synth.ALPHA_ACT, O.ACT_U4)
+    assert np.float32(step) == st_ref
+    _, _, _, y_ref = O.layer_conv(Wt, scheme, bits, alpha, codes, st_ref, 1, 1)
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.reshape(N, L.M).view(np.uint32))
