@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the RMSMP layer path on B200.
+
+Workload: the 19 3x3/1x1 convolutions of ResNet-18 at 224x224 input, batch 256 per GPU, run
+layer by layer; every layer has its own seeded Kaiming weights (rows assigned PoT-4 : Fixed-4 :
+Fixed-8 = 60:35:5 by variance rank) and its own seeded half-normal fp32 NHWC input.  One step is
+one pass of the whole path over that batch: for every layer quantize+pack the fp32 weights,
+quantize the fp32 activations to 4-bit codes, run the mixed-scheme implicit-GEMM convolution
+(int32 accumulate, per-row scaled fp32 output).  Operations are counted as 2 per multiply-
+accumulate (the convention of the paper's Table 6).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2111_00153_b200 import synth  # noqa: E402
+
+METRIC = "mixed_scheme_gemm_tops"
+UNIT = "TOPS"
+RATIO = synth.RATIO_RMSMP1
+BATCH = 256
+WORKLOAD = "resnet18_conv_stack_3x3_1x1_224px_batch256_ratio60:35:5"
+
+
+def layer_list():
+    out = []
+    for L in synth.resnet18_convs():
+        for _ in range(L.count):
+            out.append(L)
+    return out
+
+
+def host_layer(idx, L, batch, rank=0):
+    g = synth.rng(4, idx + 100 * rank)
+    W = synth.weights_kaiming(g, L.M, L.Cin, L.k, L.k)
+    x = synth.act_halfnormal(g, (batch, L.H, L.H, L.Cin))
+    return W, x
+
+
+def layer_ops(L, batch):
+    return 2 * L.macs(batch)
+
+
+def layer_alg_bytes(L, batch, nP, nF4, n8):
+    """Algorithmic bytes of one convolution launch: packed codes + 8 B/row metadata + each
+    activation code the layer needs once (a strided 1x1 needs only the sampled pixels) + fp32 out."""
+    K = L.K
+    w = (nP + nF4) * K // 2 + n8 * K + 8 * L.M
+    pix_in = L.Ho * L.Ho if (L.k == 1 and L.stride > 1) else L.H * L.H
+    a = batch * pix_in * L.Cin
+    o = 4 * batch * L.Ho * L.Ho * L.M
+    return w + a + o
+
+
+# ---------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.idx = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, smax, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); smax.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if not sm:
+            return None
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2111_00153_b200 import binding as R
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    R.lib()
+
+    layers = layer_list()
+    batch = args.batch
+    stream = torch.cuda.current_stream()
+
+    # ---- host inputs (seeded, synthetic) and device buffers
+    H = []
+    for i, L in enumerate(layers):
+        W, x = host_layer(i, L, batch, rank)
+        scheme, bits = R.rmsmp_assign_rows(W, RATIO)        # offline decision, not timed
+        alpha = synth.alpha_rows(W)
+        lay = R.rmsmp_layer_init(L.M, L.Cin, L.k, L.k, scheme, bits)
+        H.append(dict(L=L, W=W, x=x, scheme=scheme, bits=bits, alpha=alpha, lay=lay))
+    D = []
+    for h in H:
+        L = h["L"]
+        N = batch * L.Ho * L.Ho
+        D.append(dict(
+            W=torch.from_numpy(h["W"]).cuda(), x=torch.from_numpy(h["x"]).cuda(),
+            packed=torch.empty(h["lay"].packed_bytes, dtype=torch.uint8, device="cuda"),
+            codes=torch.empty(h["x"].shape, dtype=torch.int8, device="cuda"),
+            y=torch.empty((N, L.M), dtype=torch.float32, device="cuda"), N=N))
+
+    def step(ev=None):
+        for i, (h, d) in enumerate(zip(H, D)):
+            L = h["L"]
+            R.rmsmp_quantize_pack(d["W"], R.W_CONV_OIHW, h["lay"], h["scheme"], h["bits"], h["alpha"],
+                                  R.POT_NEAREST, d["packed"], stream=stream)
+            st = R.rmsmp_quantize_act(d["x"], d["x"].numel(), synth.ALPHA_ACT, R.ACT_U4, d["codes"], stream=stream)
+            if ev is not None:
+                ev[i][0].record(stream)
+            R.rmsmp_conv_implicit(h["lay"], d["packed"], d["codes"], batch, L.H, L.H, L.stride, L.pad, st,
+                                  d["y"], R.OUT_NM, None, stream=stream)
+            if ev is not None:
+                ev[i][1].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    for d in D:
+        assert R.rmsmp_last_device_status(d["packed"]) == R.OK
+
+    # ---- device-resident timing
+    evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers]
+           for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for k in range(args.steps):
+        step(evs[k])
+    t1.record(stream)
+    barrier()
+    ms_total = t0.elapsed_time(t1)
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    ops_step = sum(layer_ops(L, batch) for L in layers)
+    conv_ms = np.array([[e[0].elapsed_time(e[1]) for e in evk] for evk in evs])   # [steps][layers]
+    conv_ms_layer = conv_ms.mean(axis=0)
+    alg = np.array([layer_alg_bytes(h["L"], batch, h["lay"].nP, h["lay"].nF4, h["lay"].n8) for h in H], dtype=np.float64)
+    conv_total_ms = float(conv_ms_layer.sum())
+    achieved_gbs = float(alg.sum() / (conv_total_ms * 1e-3) / 1e9)
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    pin = []
+    for h, d in zip(H, D):
+        pin.append(dict(W=torch.from_numpy(h["W"]).pin_memory(), x=torch.from_numpy(h["x"]).pin_memory(),
+                        y=torch.empty(d["y"].shape, dtype=torch.float32).pin_memory()))
+
+    def step_e2e():
+        for h, d, p in zip(H, D, pin):
+            L = h["L"]
+            d["W"].copy_(p["W"], non_blocking=True)
+            d["x"].copy_(p["x"], non_blocking=True)
+            R.rmsmp_quantize_pack(d["W"], R.W_CONV_OIHW, h["lay"], h["scheme"], h["bits"], h["alpha"],
+                                  R.POT_NEAREST, d["packed"], stream=stream)
+            st = R.rmsmp_quantize_act(d["x"], d["x"].numel(), synth.ALPHA_ACT, R.ACT_U4, d["codes"], stream=stream)
+            R.rmsmp_conv_implicit(h["lay"], d["packed"], d["codes"], batch, L.H, L.H, L.stride, L.pad, st,
+                                  d["y"], R.OUT_NM, None, stream=stream)
+            p["y"].copy_(d["y"], non_blocking=True)
+
+    step_e2e()
+    barrier()
+    t0.record(stream)
+    for _ in range(e2e_steps):
+        step_e2e()
+    t1.record(stream)
+    barrier()
+    e2e_ms = t0.elapsed_time(t1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_ms_step = e2e_ms / e2e_steps
+    h2d = int(sum(p["W"].numel() * 4 + p["x"].numel() * 4 for p in pin))
+    d2h = int(sum(p["y"].numel() * 4 for p in pin))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_src = load_peaks()
+    out = {
+        "metric": METRIC, "value": world * ops_step / (ms_step * 1e-3) / 1e12, "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8xint8->int32 (w4/w8 a4), fp32 scale",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch_per_gpu": batch, "layers": len(layers),
+                   "ops_per_step_per_gpu": ops_step, "l2": "inputs larger than L2 (every layer reads 13-205 MB and writes 6-205 MB)",
+                   "step": "per layer: quantize_pack + quantize_act + conv_implicit (tensor variant)"},
+        "clocks": clocks,
+        "e2e": {"value": world * ops_step / (e2e_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_step,
+                "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": args.steps * len(layers) * 3,
+        "roofline": {"bound": "hbm", "kernel": "tensor_kernel (conv_implicit)", "achieved": achieved_gbs,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved_gbs / peaks["hbm_gbs"],
+                     "peak_source": peak_src, "traffic": TRAFFIC_PER_STEP_BYTES,
+                     "algorithmic_bytes_per_step": float(alg.sum()), "kernel_ms_per_step": conv_total_ms,
+                     "kernel_tops": ops_step / (conv_total_ms * 1e-3) / 1e12},
+        "per_layer": [{"name": h["L"].name, "M": h["L"].M, "K": h["L"].K, "N": d["N"], "ms": float(ms),
+                       "tops": layer_ops(h["L"], batch) / (ms * 1e-3) / 1e12, "gbs": float(a / (ms * 1e-3) / 1e9)}
+                      for h, d, ms, a in zip(H, D, conv_ms_layer, alg)],
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(args.cpu_sample_batch)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# dram bytes (read + write) of the convolution kernels of one step, from an ncu capture; None
+# until measured for the current kernel.
+TRAFFIC_PER_STEP_BYTES = None
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"])}, "of measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "of fallback"
+
+
+# ---------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_pass(batch, layers=None):
+    """One pass of the oracle over the layer stack at `batch` images; returns (seconds, ops)."""
+    from oracle import rmsmp_oracle as O
+    layers = layers or layer_list()
+    prepared = []
+    for i, L in enumerate(layers):
+        W, x = host_layer(i, L, batch)
+        scheme, bits = O.assign_rows(W, RATIO)
+        prepared.append((L, W, x, scheme, bits, synth.alpha_rows(W)))
+    t0 = time.perf_counter()
+    for L, W, x, scheme, bits, alpha in prepared:
+        codes, st = O.quantize_act(x, synth.ALPHA_ACT, O.ACT_U4)
+        O.layer_conv(W, scheme, bits, alpha, codes, st, L.stride, L.pad)
+    dt = time.perf_counter() - t0
+    return dt, sum(layer_ops(L, batch) for L in layers)
+
+
+def cpu_baseline(sample_batch):
+    from oracle import rmsmp_oracle as O
+    O.build()
+    oracle_pass(1)                       # page in / warm
+    dt, ops = oracle_pass(sample_batch)
+    return {"value": ops / dt / 1e12, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": "the same 19-layer stack at batch %d of %d (%.1f s)" % (sample_batch, BATCH, dt)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import rmsmp_oracle as O
+    O.build()
+    t1, _ = oracle_pass(1)
+    t1, _ = oracle_pass(1)
+    n = args.steps + args.warmup
+    b = int(max(1, min(32, 150.0 / (n * max(t1, 1e-3)))))
+    for _ in range(args.warmup):
+        oracle_pass(b)
+    tot, ops = 0.0, 0
+    for _ in range(args.steps):
+        dt, o = oracle_pass(b)
+        tot += dt
+        ops += o
+    val = ops / tot / 1e12
+    sample = "the same 19-layer stack at batch %d of %d per step" % (b, BATCH)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8xint8->int32 (w4/w8 a4), fp32 scale", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=BATCH)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-sample-batch", type=int, default=32)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
