@@ -38,9 +38,16 @@ BATCH = 256
 WORKLOAD = "resnet18_conv_stack_3x3_1x1_224px_batch256_ratio60:35:5"
 
 
+LAYER_FILTER = None    # set by --layers: comma-separated layer names, one instance each
+
+
 def layer_list():
     out = []
     for L in synth.resnet18_convs():
+        if LAYER_FILTER is not None:
+            if L.name in LAYER_FILTER:
+                out.append(L)
+            continue
         for _ in range(L.count):
             out.append(L)
     return out
@@ -212,8 +219,10 @@ def run_ours(args):
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    if args.no_e2e:
+        e2e_steps = 0
     pin = []
-    for h, d in zip(H, D):
+    for h, d in zip(H, D) if e2e_steps else ():
         pin.append(dict(W=torch.from_numpy(h["W"]).pin_memory(), x=torch.from_numpy(h["x"]).pin_memory(),
                         y=torch.empty(d["y"].shape, dtype=torch.float32).pin_memory()))
 
@@ -229,7 +238,8 @@ def run_ours(args):
                                   d["y"], R.OUT_NM, None, stream=stream)
             p["y"].copy_(d["y"], non_blocking=True)
 
-    step_e2e()
+    if e2e_steps:
+        step_e2e()
     barrier()
     t0.record(stream)
     for _ in range(e2e_steps):
@@ -241,7 +251,7 @@ def run_ours(args):
         t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
-    e2e_ms_step = e2e_ms / e2e_steps
+    e2e_ms_step = e2e_ms / max(e2e_steps, 1)
     h2d = int(sum(p["W"].numel() * 4 + p["x"].numel() * 4 for p in pin))
     d2h = int(sum(p["y"].numel() * 4 for p in pin))
 
@@ -256,12 +266,12 @@ def run_ours(args):
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8xint8->int32 (w4/w8 a4), fp32 scale",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD, "batch_per_gpu": batch, "layers": len(layers),
+        "config": {"workload": WORKLOAD if LAYER_FILTER is None else "subset:" + ",".join(sorted(LAYER_FILTER)), "batch_per_gpu": batch, "layers": len(layers),
                    "ops_per_step_per_gpu": ops_step, "l2": "inputs larger than L2 (every layer reads 13-205 MB and writes 6-205 MB)",
                    "step": "per layer: quantize_pack + quantize_act + conv_implicit (tensor variant)"},
         "clocks": clocks,
-        "e2e": {"value": world * ops_step / (e2e_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_step,
-                "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": ({"value": world * ops_step / (e2e_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_step,
+                 "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h} if e2e_steps else None),
         "gpu_launches": args.steps * len(layers) * 3,
         "roofline": {"bound": "hbm", "kernel": "tensor_kernel (conv_implicit)", "achieved": achieved_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved_gbs / peaks["hbm_gbs"],
@@ -360,9 +370,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=BATCH)
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-sample-batch", type=int, default=32)
+    ap.add_argument("--cpu-sample-batch", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--layers", default=None,
+                    help="comma-separated layer names: run one instance of each (profiling runs)")
     args = ap.parse_args()
+    if args.layers:
+        global LAYER_FILTER
+        LAYER_FILTER = set(args.layers.split(","))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -21,6 +21,7 @@
 // RMSMP_ERR_TIMEOUT in the packed buffer's status word, all roles leave their loops, tensor
 // memory is freed and the kernel returns.
 #include <cuda.h>
+#include <cstring>
 #include "common.cuh"
 #include "decode.cuh"
 
@@ -34,7 +35,9 @@ constexpr int kABytes = kBlockRows * 128;        // 16 KB: 128 rows x 128 B (one
 constexpr int kBBytes = kTileN * 128;            // 32 KB
 constexpr int kNumExpWarps = 8;
 constexpr int kThreads = 32 * (2 + kNumExpWarps + 4);
-constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kEpiFirstThread = 32 * (2 + kNumExpWarps);   // issues the bulk stores
+constexpr int kStageOut = 32 * kBlockRows * 4;   // 16 KB: one 32-pixel x 128-row fp32/int32 output chunk
+constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + 2 * kStageOut + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 struct TensorCfg {
@@ -48,6 +51,12 @@ struct TensorCfg {
     int nkb;               // k-blocks per tile = taps * cpt
     uint32_t idesc;
     uint32_t tx_bytes;     // bytes one activation box brings
+    int tma_store;         // 1: output chunks leave through shared memory and bulk tensor stores
+    int tail_rows;         // npix % 32: height of the last chunk of a tile (0: none)
+};
+
+struct StoreMaps {         // bulk-store tensor maps: fp32 output and int32 accumulators, full and tail chunk
+    CUtensorMap out_full, out_tail, acc_full, acc_tail;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -114,6 +123,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
@@ -234,18 +251,21 @@ __device__ __forceinline__ void exp_store(const RawBuf& r, uint32_t a_stage, int
 // ------------------------------------------------------------------ the kernel
 
 __global__ void __launch_bounds__(kThreads, 1)
-tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUtensorMap act_map)
+tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUtensorMap act_map,
+              const __grid_constant__ StoreMaps smaps)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sA = smem_base;
     const uint32_t sB = smem_base + kStages * kABytes;
-    const uint32_t sBar = sB + kStages * kBBytes;
+    const uint32_t sOut = sB + kStages * kBBytes;
+    const uint32_t sBar = sOut + 2 * kStageOut;
     // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]
     const uint32_t bar_full = sBar, bar_empty = sBar + 8 * kStages;
     const uint32_t bar_tfull = sBar + 16 * kStages, bar_tempty = bar_tfull + 16;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ int s_epi_stop;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -379,7 +399,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
     } else {
         // ---------------------------------------------------------- epilogue
         const int quarter = warp & 3;              // TMEM lanes this warp may read
-        uint32_t it = 0;
+        uint32_t it = 0, stg_count = 0;
         for (int64_t tile = first; tile < cfg.ntiles; tile += step, ++it) {
             const uint32_t ab = it & 1;
             const int blk = (int)(tile % p.nblocks);
@@ -396,9 +416,71 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
                 scale = __fmul_rn(__ldg(p.wstep + m), p.act_step);
                 shift = (__ldg(p.kind + m) == kFixed4) ? 4 : 0;
             }
-            if (!mbar_wait_warp(bar_tfull + 8 * ab, (it >> 1) & 1, abort_flag)) break;
+            const bool got = mbar_wait_warp(bar_tfull + 8 * ab, (it >> 1) & 1, abort_flag);
+            if (cfg.tma_store) {
+                // the four epilogue warps meet at named barriers below: leave together or not at all
+                epi_bar();
+                if (threadIdx.x == kEpiFirstThread) s_epi_stop = *abort_flag;
+                epi_bar();
+                if (s_epi_stop) break;
+            } else if (!got) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * kTileN;
+            if (cfg.tma_store) {
+                const int m_local = quarter * 32 + lane;
+                const int nchunks = (nvalid + 31) >> 5;
+                for (int c = 0; c < nchunks; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c * 32, v);
+                    if (c == nchunks - 1) {
+                        // all accumulators of this tile are in registers: hand the buffer back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
+                    }
+                    const bool tail = cfg.tail_rows && (c == (cfg.npix >> 5));
+                    const int nsub = p.acc ? 2 : 1;
+                    for (int sub = 0; sub < nsub; ++sub) {
+                        const uint32_t stg = sOut + (stg_count & 1) * kStageOut;
+                        ++stg_count;
+                        epi_bar();                       // the buffer's previous store has been read out
+                        if (!p.out_mn) {
+                            // [pixel][row] : a warp writes 128 contiguous bytes per pixel
+                            const uint32_t a0 = stg + m_local * 4;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const int a = (int)v[j] >> shift;
+                                const uint32_t w = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
+                                asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 512), "r"(w) : "memory");
+                            }
+                        } else {
+                            // [row][pixel], 16-byte chunks swizzled by row (matches the 128-byte-swizzled store map)
+                            const uint32_t a0 = stg + m_local * 128;
+#pragma unroll
+                            for (int cc = 0; cc < 8; ++cc) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) {
+                                    const int a = (int)v[4 * cc + t] >> shift;
+                                    w[t] = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
+                                }
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                             ::"r"(a0 + ((cc ^ (m_local & 7)) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+                            }
+                        }
+                        fence_proxy_async_smem();
+                        epi_bar();                       // chunk complete in shared memory
+                        if (threadIdx.x == kEpiFirstThread) {
+                            const CUtensorMap* map = sub ? (tail ? &smaps.acc_tail : &smaps.acc_full)
+                                                         : (tail ? &smaps.out_tail : &smaps.out_full);
+                            const int cm = blk * kBlockRows, cn = (int)(n0 + c * 32);
+                            if (!p.out_mn) tma_store_2d(map, stg, cm, cn); else tma_store_2d(map, stg, cn, cm);
+                            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        }
+                    }
+                }
+                continue;
+            }
             for (int c = 0; c * 32 < nvalid; ++c) {
                 uint32_t v[32];
                 tmem_ld32(taddr + c * 32, v);
@@ -451,6 +533,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
     }
 
     // ---------------------------------------------------------- teardown
+    if (threadIdx.x == kEpiFirstThread) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -541,6 +624,36 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return RMSMP_ERR_CUDA;
 
+    StoreMaps sm;
+    memset(&sm, 0, sizeof(sm));
+    c.tma_store = 0;
+    c.tail_rows = c.npix & 31;
+    const bool ld_ok = (p.ld_out % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
+                       (!p.acc || (reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
+    if (ld_ok && (!p.out_mn || c.tail_rows == 0)) {
+        auto make = [&](CUtensorMap* m, void* base, CUtensorMapDataType dt, int rows) -> bool {
+            if (!p.out_mn) {
+                const cuuint64_t gd[2] = {(cuuint64_t)p.M, (cuuint64_t)p.N};
+                const cuuint64_t gs[1] = {(cuuint64_t)p.ld_out * 4};
+                const cuuint32_t bx[2] = {(cuuint32_t)kBlockRows, (cuuint32_t)rows};
+                const cuuint32_t es[2] = {1, 1};
+                return enc(m, dt, 2, base, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                           CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            }
+            const cuuint64_t gd[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
+            const cuuint64_t gs[1] = {(cuuint64_t)p.ld_out * 4};
+            const cuuint32_t bx[2] = {32u, (cuuint32_t)kBlockRows};
+            const cuuint32_t es[2] = {1, 1};
+            return enc(m, dt, 2, base, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        };
+        bool ok = make(&sm.out_full, p.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 32);
+        if (ok && c.tail_rows) ok = make(&sm.out_tail, p.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.tail_rows);
+        if (ok && p.acc) ok = make(&sm.acc_full, p.acc, CU_TENSOR_MAP_DATA_TYPE_INT32, 32);
+        if (ok && p.acc && c.tail_rows) ok = make(&sm.acc_tail, p.acc, CU_TENSOR_MAP_DATA_TYPE_INT32, c.tail_rows);
+        c.tma_store = ok ? 1 : 0;
+    }
+
     static int sm_count = 0;
     static bool attr_set = false;
     if (!attr_set) {
@@ -554,7 +667,7 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
         attr_set = true;
     }
     const int grid = (int)std::min<int64_t>(c.ntiles, sm_count > 0 ? sm_count : 148);
-    tensor_kernel<<<grid, kThreads, kSmemBytes, st>>>(p, c, map);
+    tensor_kernel<<<grid, kThreads, kSmemBytes, st>>>(p, c, map, sm);
     if (cudaGetLastError() != cudaSuccess) return RMSMP_ERR_CUDA;
     return RMSMP_OK;
 }
