@@ -205,6 +205,20 @@ rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* layer, const void* d
  */
 rmsmp_status rmsmp_last_device_status(const void* d_packed, void* stream);
 
+/*
+ * Measurement helper (no counterpart in the paper): the tensor-pipe ceiling of the current GPU
+ * for the MMA shape the contraction kernel issues (M=128, N=n_cols, operands resident in shared
+ * memory, every SM busy, no loads or stores).  use_bf16 = 0 measures kind::i8 (the INT8 roofline
+ * the layer kernels are reported against), 1 measures bf16 for calibration.  Runs `iters`
+ * k-blocks of 4 instructions per SM, synchronises, writes tera-operations per second
+ * (2 ops per multiply-accumulate) to *h_tops and the duration to *h_ms (may be NULL).
+ * d_status_word: 4 bytes of device memory the kernel may record a wait time-out in.
+ * Errors: NULL, SHAPE (iters outside 1..2^22, n_cols not a multiple of 16 in 16..256), ARCH,
+ * CUDA, TIMEOUT.
+ */
+rmsmp_status rmsmp_measure_mma_peak(int use_bf16, int n_cols, int iters, uint32_t* d_status_word,
+                                    float* h_tops, float* h_ms, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,6 +29,7 @@ EXPORTS = (
     "rmsmp_status_string", "rmsmp_assign_rows", "rmsmp_layer_init", "rmsmp_quantize_pack",
     "rmsmp_unpack_codes", "rmsmp_quantize_act", "rmsmp_gemm", "rmsmp_gemm_variant",
     "rmsmp_conv_implicit", "rmsmp_conv_implicit_variant", "rmsmp_last_device_status",
+    "rmsmp_measure_mma_peak",
 )
 
 
@@ -89,6 +90,7 @@ def lib() -> C.CDLL:
         L.rmsmp_conv_implicit_variant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i32, i32, i32,
                                                   i32, i32, f32, vp, i32, vp, i32, vp]
         L.rmsmp_last_device_status.argtypes = [vp, vp]
+        L.rmsmp_measure_mma_peak.argtypes = [i32, i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
         _lib = L
     return _lib
 
@@ -206,3 +208,13 @@ def rmsmp_conv_implicit_variant(layer, d_packed, d_act, B: int, H: int, W: int, 
 
 def rmsmp_last_device_status(d_packed, stream=None) -> int:
     return lib().rmsmp_last_device_status(_dp(d_packed), _stream(stream))
+
+
+def rmsmp_measure_mma_peak(d_status_word, use_bf16: bool = False, n_cols: int = 256,
+                           iters: int = 20000, stream=None):
+    """Tensor-pipe ceiling for the kernel's MMA shape: returns (tera-ops per second, milliseconds)."""
+    tops, ms = C.c_float(0.0), C.c_float(0.0)
+    _check(lib().rmsmp_measure_mma_peak(1 if use_bf16 else 0, n_cols, iters, _dp(d_status_word),
+                                        C.byref(tops), C.byref(ms), _stream(stream)),
+           "rmsmp_measure_mma_peak")
+    return tops.value, ms.value
