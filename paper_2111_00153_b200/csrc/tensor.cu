@@ -15,7 +15,7 @@
 //               fetched group by group (PoT, Fixed-4, Fixed-8) but written to the row position
 //               of their ORIGINAL index, so accumulator lanes are in original row order and
 //               the output needs no scatter.
-//   warps 10-13 epilogue: tcgen05.ld the accumulators, undo the x16 of Fixed-4 rows, convert,
+//   warps 10+   epilogue: tcgen05.ld the accumulators, undo the x16 of Fixed-4 rows, convert,
 //               scale by wstep*act_step, store.
 // Every wait on an mbarrier is bounded; when one runs out the kernel records
 // RMSMP_ERR_TIMEOUT in the packed buffer's status word, all roles leave their loops, tensor
@@ -34,10 +34,12 @@ constexpr int kTileN = 256;                      // pixels per tile (max) = TMEM
 constexpr int kABytes = kBlockRows * 128;        // 16 KB: 128 rows x 128 B (one k-block)
 constexpr int kBBytes = kTileN * 128;            // 32 KB
 constexpr int kNumExpWarps = 8;
-constexpr int kThreads = 32 * (2 + kNumExpWarps + 4);
-constexpr int kEpiFirstThread = 32 * (2 + kNumExpWarps);   // issues the bulk stores
-constexpr int kStageOut = 32 * kBlockRows * 4;   // 16 KB: one 32-pixel x 128-row fp32/int32 output chunk
-constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + 2 * kStageOut + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kNumEpiWarps = 4;                 // kEpiPerQuarter warps share a tensor-memory quarter, alternating 32-pixel chunks
+constexpr int kEpiPerQuarter = kNumEpiWarps / 4;
+constexpr int kThreads = 32 * (2 + kNumExpWarps + kNumEpiWarps);
+constexpr int kWarpStage = 32 * 32 * 4;          // 4 KB: 32 pixels x 32 rows of fp32/int32, one epilogue warp's chunk
+constexpr int kStageOut = kNumEpiWarps * kWarpStage;   // one private buffer per epilogue warp
+constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + kStageOut + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 struct TensorCfg {
@@ -130,7 +132,6 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
                  ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
@@ -259,13 +260,12 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
     const uint32_t sA = smem_base;
     const uint32_t sB = smem_base + kStages * kABytes;
     const uint32_t sOut = sB + kStages * kBBytes;
-    const uint32_t sBar = sOut + 2 * kStageOut;
+    const uint32_t sBar = sOut + kStageOut;
     // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]
     const uint32_t bar_full = sBar, bar_empty = sBar + 8 * kStages;
     const uint32_t bar_tfull = sBar + 16 * kStages, bar_tempty = bar_tfull + 16;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ int s_epi_stop;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -276,7 +276,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_tfull + 8 * b, 1);                  // tcgen05.commit
-            mbar_init(bar_tempty + 8 * b, 4);                 // one arrival per epilogue warp
+            mbar_init(bar_tempty + 8 * b, kNumEpiWarps);      // one arrival per epilogue warp
         }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -399,7 +399,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
     } else {
         // ---------------------------------------------------------- epilogue
         const int quarter = warp & 3;              // TMEM lanes this warp may read
-        uint32_t it = 0, stg_count = 0;
+        const int half = (warp - (2 + kNumExpWarps)) >> 2;   // which chunks of a tile: even or odd
+        uint32_t it = 0;
         for (int64_t tile = first; tile < cfg.ntiles; tile += step, ++it) {
             const uint32_t ab = it & 1;
             const int blk = (int)(tile % p.nblocks);
@@ -416,23 +417,29 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
                 scale = __fmul_rn(__ldg(p.wstep + m), p.act_step);
                 shift = (__ldg(p.kind + m) == kFixed4) ? 4 : 0;
             }
-            const bool got = mbar_wait_warp(bar_tfull + 8 * ab, (it >> 1) & 1, abort_flag);
-            if (cfg.tma_store) {
-                // the four epilogue warps meet at named barriers below: leave together or not at all
-                epi_bar();
-                if (threadIdx.x == kEpiFirstThread) s_epi_stop = *abort_flag;
-                epi_bar();
-                if (s_epi_stop) break;
-            } else if (!got) break;
+            if (!mbar_wait_warp(bar_tfull + 8 * ab, (it >> 1) & 1, abort_flag)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * kTileN;
             if (cfg.tma_store) {
-                const int m_local = quarter * 32 + lane;
+                // The warps of a tensor-memory quarter take alternate 32-pixel chunks of its 32 rows; each
+                // stages its chunk in a private buffer and issues its own bulk store, so no epilogue
+                // warp ever waits for another.
+                if (blk * kBlockRows + quarter * 32 >= p.M) {      // no valid row in this quarter
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
+                    continue;
+                }
+                const uint32_t stg = sOut + (uint32_t)(warp - (2 + kNumExpWarps)) * kWarpStage;
                 const int nchunks = (nvalid + 31) >> 5;
-                for (int c = 0; c < nchunks; ++c) {
+                if (half >= nchunks) {                             // a one-chunk tile leaves the odd warps idle
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
+                    continue;
+                }
+                for (int c = half; c < nchunks; c += kEpiPerQuarter) {
                     uint32_t v[32];
                     tmem_ld32(taddr + c * 32, v);
-                    if (c == nchunks - 1) {
+                    if (c + kEpiPerQuarter >= nchunks) {
                         // all accumulators of this tile are in registers: hand the buffer back
                         tc_fence_before();
                         __syncwarp();
@@ -441,21 +448,20 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
                     const bool tail = cfg.tail_rows && (c == (cfg.npix >> 5));
                     const int nsub = p.acc ? 2 : 1;
                     for (int sub = 0; sub < nsub; ++sub) {
-                        const uint32_t stg = sOut + (stg_count & 1) * kStageOut;
-                        ++stg_count;
-                        epi_bar();                       // the buffer's previous store has been read out
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();                    // the buffer's previous store has been read out
                         if (!p.out_mn) {
-                            // [pixel][row] : a warp writes 128 contiguous bytes per pixel
-                            const uint32_t a0 = stg + m_local * 4;
+                            // [pixel][row]: the warp writes 128 contiguous bytes per pixel
+                            const uint32_t a0 = stg + lane * 4;
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
                                 const int a = (int)v[j] >> shift;
                                 const uint32_t w = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
-                                asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 512), "r"(w) : "memory");
+                                asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 128), "r"(w) : "memory");
                             }
                         } else {
                             // [row][pixel], 16-byte chunks swizzled by row (matches the 128-byte-swizzled store map)
-                            const uint32_t a0 = stg + m_local * 128;
+                            const uint32_t a0 = stg + lane * 128;
 #pragma unroll
                             for (int cc = 0; cc < 8; ++cc) {
                                 uint32_t w[4];
@@ -465,17 +471,16 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
                                     w[t] = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
                                 }
                                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                                             ::"r"(a0 + ((cc ^ (m_local & 7)) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+                                             ::"r"(a0 + ((cc ^ (lane & 7)) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
                             }
                         }
                         fence_proxy_async_smem();
-                        epi_bar();                       // chunk complete in shared memory
-                        if (threadIdx.x == kEpiFirstThread) {
+                        __syncwarp();                    // chunk complete in shared memory
+                        if (lane == 0) {
                             const CUtensorMap* map = sub ? (tail ? &smaps.acc_tail : &smaps.acc_full)
                                                          : (tail ? &smaps.out_tail : &smaps.out_full);
-                            const int cm = blk * kBlockRows, cn = (int)(n0 + c * 32);
+                            const int cm = blk * kBlockRows + quarter * 32, cn = (int)(n0 + c * 32);
                             if (!p.out_mn) tma_store_2d(map, stg, cm, cn); else tma_store_2d(map, stg, cn, cm);
-                            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                         }
                     }
                 }
@@ -533,7 +538,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
     }
 
     // ---------------------------------------------------------- teardown
-    if (threadIdx.x == kEpiFirstThread) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (warp >= 2 + kNumExpWarps && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -635,14 +640,14 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
             if (!p.out_mn) {
                 const cuuint64_t gd[2] = {(cuuint64_t)p.M, (cuuint64_t)p.N};
                 const cuuint64_t gs[1] = {(cuuint64_t)p.ld_out * 4};
-                const cuuint32_t bx[2] = {(cuuint32_t)kBlockRows, (cuuint32_t)rows};
+                const cuuint32_t bx[2] = {32u, (cuuint32_t)rows};
                 const cuuint32_t es[2] = {1, 1};
                 return enc(m, dt, 2, base, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
             }
             const cuuint64_t gd[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
             const cuuint64_t gs[1] = {(cuuint64_t)p.ld_out * 4};
-            const cuuint32_t bx[2] = {32u, (cuuint32_t)kBlockRows};
+            const cuuint32_t bx[2] = {32u, 32u};
             const cuuint32_t es[2] = {1, 1};
             return enc(m, dt, 2, base, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                        CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
