@@ -39,7 +39,7 @@ class rmsmp_layer(C.Structure):
         ("M", C.c_int32), ("Cin", C.c_int32), ("kh", C.c_int32), ("kw", C.c_int32),
         ("Cp", C.c_int32), ("Kp", C.c_int32),
         ("nP", C.c_int32), ("nF4", C.c_int32), ("n8", C.c_int32),
-        ("nblocks", C.c_int32), ("reserved", C.c_int32),
+        ("nblocks", C.c_int32), ("raw_stage_bytes", C.c_int32),
         ("off_perm", C.c_uint64), ("off_slot", C.c_uint64), ("off_wstep", C.c_uint64),
         ("off_alpha", C.c_uint64), ("off_kind", C.c_uint64), ("off_blocks", C.c_uint64),
         ("off_q4", C.c_uint64), ("off_q8", C.c_uint64),

@@ -36,7 +36,7 @@ struct Problem {
     const uint8_t* q4;        // [(nP+nF4)][Kp/2]
     const uint8_t* q8;        // [n8][Kp]
     uint32_t* status;
-    int M, Cin, kh, kw, Cp, Kp, nP, nF4, n8, nblocks;
+    int M, Cin, kh, kw, Cp, Kp, nP, nF4, n8, nblocks, raw_stage_bytes;
     // activations: [B][H][W] pixels of `pix_pitch` bytes, Cin codes used in each
     const int8_t* act;
     int B, H, W, Ho, Wo, stride, pad;

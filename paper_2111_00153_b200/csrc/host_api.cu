@@ -60,6 +60,7 @@ void fill_problem(Problem& p, const rmsmp_layer* L, const void* d_packed)
     p.status = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(blob) + kStatusOffset);
     p.M = L->M; p.Cin = L->Cin; p.kh = L->kh; p.kw = L->kw; p.Cp = L->Cp; p.Kp = L->Kp;
     p.nP = L->nP; p.nF4 = L->nF4; p.n8 = L->n8; p.nblocks = L->nblocks;
+    p.raw_stage_bytes = L->raw_stage_bytes;
 }
 
 rmsmp_status dispatch(Problem& p, rmsmp_variant variant, cudaStream_t st)
@@ -158,6 +159,15 @@ rmsmp_status rmsmp_layer_init(rmsmp_layer* L, int M, int Cin, int kh, int kw,
     if (kh * kw > 1 && L->Kp > 196608) return RMSMP_ERR_SHAPE;   // one shared-memory segment in the pack kernel
     L->nP = cnt[0]; L->nF4 = cnt[1]; L->n8 = cnt[2];
     L->nblocks = (M + kBlockRows - 1) / kBlockRows;
+    // bytes one k-block of one block's packed rows takes when fetched group by group in 16-row boxes
+    int raw_max = 0;
+    for (int b0 = 0; b0 < M; b0 += kBlockRows) {
+        int c[3] = {0, 0, 0};
+        for (int r = b0; r < M && r < b0 + kBlockRows; ++r) ++c[row_kind(h_scheme[r], h_bits[r])];
+        const int bytes = ((c[0] + 15) / 16 * 16 + (c[1] + 15) / 16 * 16) * 64 + (c[2] + 15) / 16 * 16 * 128;
+        raw_max = std::max(raw_max, bytes);
+    }
+    L->raw_stage_bytes = raw_max;
     uint64_t off = 256;
     L->off_perm = off;   off = align_up(off + 4ull * M, 256);
     L->off_slot = off;   off = align_up(off + 4ull * M, 256);

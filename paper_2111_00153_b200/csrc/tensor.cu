@@ -1,22 +1,25 @@
 // Tensor-core variant of the contraction for sm_100a.
 //
-// One persistent CTA per SM walks over output tiles of 128 weight rows x up to 256 pixels.
-// Warp roles:
-//   warp 0      TMA producer: activation-code tiles (the B operand) global -> shared memory,
-//               128-byte swizzled, one 4-D box per k-block; for a convolution the box is the
-//               window of input pixels one filter tap needs (zero fill outside the image = the
-//               padding), so no im2col buffer exists anywhere.
-//   warp 1      allocates tensor memory, issues tcgen05.mma (kind::i8, int32 accumulators in
-//               tensor memory, two 256-column buffers so tile i+1 is computed while tile i
-//               is being written out).
-//   warps 2-9   expanders: fetch the packed 4-bit / 8-bit weight codes of the tile's rows,
-//               expand them to int8 in registers and store them into shared memory in the
-//               K-major 128-byte-swizzled layout the MMA reads (the A operand).  Rows are
-//               fetched group by group (PoT, Fixed-4, Fixed-8) but written to the row position
-//               of their ORIGINAL index, so accumulator lanes are in original row order and
-//               the output needs no scatter.
-//   warps 10+   epilogue: tcgen05.ld the accumulators, undo the x16 of Fixed-4 rows, convert,
-//               scale by wstep*act_step, store.
+// One persistent CTA per SM walks over output tiles of 128 weight rows x up to 256 pixels; the
+// reduction is cut into k-blocks of 128 codes.  Warp roles:
+//   warp 0      TMA producer.  Per k-block it fetches (a) the activation-code tile (the B
+//               operand): one 4-D box into 128-byte-swizzled shared memory -- for a convolution
+//               the box is the window of input pixels one filter tap needs, zero fill outside the
+//               image being the padding, so no im2col buffer exists anywhere; (b) the packed
+//               4-bit / 8-bit weight codes of the tile's rows, as 16-row boxes, into a raw ring.
+//   warp 1      allocates tensor memory and issues tcgen05.mma (kind::i8, int32 accumulators in
+//               tensor memory, two 256-column buffers: tile i+1 is computed while tile i is
+//               written out).
+//   warps 2-9   expanders, two groups of four warps that take alternate k-blocks: read the raw
+//               codes from shared memory, expand them to int8 in registers and store them in the
+//               K-major 128-byte-swizzled layout the MMA reads (the A operand).  Rows arrive
+//               group by group (PoT, Fixed-4, Fixed-8) but are written to the row of their ORIGINAL
+//               index, so accumulator lanes are in original row order and the output needs no
+//               scatter through the permutation.
+//   warps 10-13 epilogue, one per tensor-memory quarter: tcgen05.ld (next chunk in flight while
+//               the current one is processed), undo the x16 of Fixed-4 rows, convert, scale by
+//               wstep*act_step, stage 32 pixels x 32 rows in a private double buffer and write it
+//               with a bulk tensor store.
 // Every wait on an mbarrier is bounded; when one runs out the kernel records
 // RMSMP_ERR_TIMEOUT in the packed buffer's status word, all roles leave their loops, tensor
 // memory is freed and the kernel returns.
@@ -29,17 +32,17 @@ namespace rmsmp {
 
 namespace {
 
-constexpr int kStages = 4;
 constexpr int kTileN = 256;                      // pixels per tile (max) = TMEM columns per buffer
 constexpr int kABytes = kBlockRows * 128;        // 16 KB: 128 rows x 128 B (one k-block)
 constexpr int kBBytes = kTileN * 128;            // 32 KB
-constexpr int kNumExpWarps = 8;
-constexpr int kNumEpiWarps = 4;                 // kEpiPerQuarter warps share a tensor-memory quarter, alternating 32-pixel chunks
-constexpr int kEpiPerQuarter = kNumEpiWarps / 4;
+constexpr int kGroups = 2;                       // expander groups taking alternate k-blocks
+constexpr int kNumExpWarps = 4 * kGroups;
+constexpr int kNumEpiWarps = 4;
 constexpr int kThreads = 32 * (2 + kNumExpWarps + kNumEpiWarps);
-constexpr int kWarpStage = 32 * 32 * 4;          // 4 KB: 32 pixels x 32 rows of fp32/int32, one epilogue warp's chunk
-constexpr int kStageOut = kNumEpiWarps * kWarpStage;   // one private buffer per epilogue warp
-constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + kStageOut + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kWarpStage = 32 * 32 * 4;          // 4 KB: 32 pixels x 32 rows of fp32/int32
+constexpr int kRawBoxRows = 16;                  // rows per raw weight box
+constexpr int kMaxRing = 8;
+constexpr int kSmemLimit = 232448 - 1024;        // 227 KB per CTA less room for the static variables
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 struct TensorCfg {
@@ -51,14 +54,21 @@ struct TensorCfg {
     int64_t ntiles;        // ntiles_n * nblocks
     int cpt;               // 128-channel chunks per tap
     int nkb;               // k-blocks per tile = taps * cpt
+    int last_ksteps;       // 32-code steps in the last chunk of a tap
     uint32_t idesc;
     uint32_t tx_bytes;     // bytes one activation box brings
     int tma_store;         // 1: output chunks leave through shared memory and bulk tensor stores
     int tail_rows;         // npix % 32: height of the last chunk of a tile (0: none)
+    int nA, nB, nR;        // ring depths: expanded weights, activations, raw weights
+    uint32_t raw_bytes;    // one raw stage
+    int out_bufs;          // staging buffers per epilogue warp (1 or 2)
+    uint32_t smem_bytes;
 };
 
-struct StoreMaps {         // bulk-store tensor maps: fp32 output and int32 accumulators, full and tail chunk
-    CUtensorMap out_full, out_tail, acc_full, acc_tail;
+struct Maps {
+    CUtensorMap act;                                   // [B][H][W][Cin] activation codes
+    CUtensorMap q4, q8;                                // packed weight regions
+    CUtensorMap out_full, out_tail, acc_full, acc_tail;   // bulk stores: 32-row and tail chunks
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -125,7 +135,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
-
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1)
 {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
@@ -159,7 +175,8 @@ __device__ __forceinline__ void mma_commit(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t v[32])
+// Issue a 32-column accumulator load; the registers are valid only after tmem_ld_wait(v).
+__device__ __forceinline__ void tmem_ld_issue(uint32_t taddr, uint32_t (&v)[32])
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -171,108 +188,109 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t v[32])
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Wait for the outstanding loads.  The registers pass through the statement so that no use of
+// them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+                   "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+                   "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+                 :: "memory");
 }
 
-// ------------------------------------------------------------------ expander state
+// ------------------------------------------------------------------ per-tile row bookkeeping
 
-// What an expander thread needs to know about one of its two rows in a tile.
-struct RowTask {
-    const uint8_t* src;   // start of the packed row (4-bit or 8-bit region)
-    int meta;             // bits 0-7: destination row in the tile, bits 8-9: kind, 3 = no row
+// Rows of one 128-row block inside the three groups of the packed buffer.
+struct BlockInfo {
+    int p0, nP, f0, nF, e0, nE;
 };
-
-__device__ __forceinline__ RowTask make_task(const Problem& p, int64_t tile, int slot_in_tile)
+__device__ __forceinline__ BlockInfo load_block(const Problem& p, int blk)
 {
-    RowTask t;
-    t.src = p.q4;
-    t.meta = 3 << 8;
-    if (tile < 0) return t;
-    const int blk = (int)(tile % p.nblocks);
     const int4 b0 = __ldg(reinterpret_cast<const int4*>(p.blocks + 8 * blk));
     const int2 b1 = __ldg(reinterpret_cast<const int2*>(p.blocks + 8 * blk + 4));
-    const int nP = b0.y, nF = b0.w, nE = b1.y;
-    int kind, packed;
-    if (slot_in_tile < nP) { kind = kPoT4; packed = b0.x + slot_in_tile; }
-    else if (slot_in_tile < nP + nF) { kind = kFixed4; packed = p.nP + b0.z + (slot_in_tile - nP); }
-    else if (slot_in_tile < nP + nF + nE) { kind = kFixed8; packed = p.nP + p.nF4 + b1.x + (slot_in_tile - nP - nF); }
-    else return t;
+    BlockInfo b;
+    b.p0 = b0.x; b.nP = b0.y; b.f0 = b0.z; b.nF = b0.w; b.e0 = b1.x; b.nE = b1.y;
+    return b;
+}
+__device__ __forceinline__ int ceil_box(int n) { return (n + kRawBoxRows - 1) / kRawBoxRows * kRawBoxRows; }
+
+// What an expander thread knows about one of its rows in a tile, in one word:
+// bits 0-15 byte offset of its 32 codes inside a raw stage, bits 16-29 byte offset of its first
+// 16-byte chunk inside an A stage (the second chunk is that offset ^ 16), bits 30-31 kind (3: none).
+__device__ __forceinline__ uint32_t make_meta(const Problem& p, int64_t tile, int slot, int q)
+{
+    if (tile < 0) return 3u << 30;
+    const int blk = (int)(tile % p.nblocks);
+    const BlockInfo b = load_block(p, blk);
+    int kind, packed, raw;
+    if (slot < b.nP) {
+        kind = kPoT4; packed = b.p0 + slot; raw = slot * 64 + q * 16;
+    } else if (slot < b.nP + b.nF) {
+        kind = kFixed4; packed = p.nP + b.f0 + (slot - b.nP);
+        raw = (ceil_box(b.nP) + slot - b.nP) * 64 + q * 16;
+    } else if (slot < b.nP + b.nF + b.nE) {
+        kind = kFixed8; packed = p.nP + p.nF4 + b.e0 + (slot - b.nP - b.nF);
+        raw = (ceil_box(b.nP) + ceil_box(b.nF)) * 64 + (slot - b.nP - b.nF) * 128 + q * 32;
+    } else {
+        return 3u << 30;
+    }
     const int row = __ldg(p.perm + packed) - blk * kBlockRows;
-    t.src = (kind == kFixed8) ? p.q8 + (size_t)(packed - p.nP - p.nF4) * p.Kp
-                              : p.q4 + (size_t)packed * (p.Kp >> 1);
-    t.meta = row | (kind << 8);
-    return t;
+    const uint32_t aoff = (uint32_t)row * 128u + ((uint32_t)((2 * q) ^ (row & 7)) << 4);
+    return (uint32_t)raw | (aoff << 16) | ((uint32_t)kind << 30);
 }
 
-struct RawBuf {
-    uint4 lo[2], hi[2];   // per task: 16 bytes (4-bit rows) or 32 bytes (8-bit rows)
-    int meta[2];
-};
-
-__device__ __forceinline__ void exp_load(RawBuf& r, const RowTask task[2], int koff, bool active)
+// Expand one task: 32 codes from the raw stage to two 16-byte chunks of the A stage.
+__device__ __forceinline__ void expand_task(uint32_t meta, uint32_t raw_stage, uint32_t a_stage)
 {
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        r.meta[j] = active ? task[j].meta : (3 << 8);
-        const int kind = (r.meta[j] >> 8) & 3;
-        if (kind == kFixed8) {
-            const uint4* s = reinterpret_cast<const uint4*>(task[j].src + koff);
-            r.lo[j] = __ldg(s);
-            r.hi[j] = __ldg(s + 1);
-        } else if (kind != 3) {
-            r.lo[j] = __ldg(reinterpret_cast<const uint4*>(task[j].src + (koff >> 1)));
-        }
+    const uint32_t kind = meta >> 30;
+    const uint32_t src = raw_stage + (meta & 0xFFFFu);
+    const uint32_t dst = a_stage + ((meta >> 16) & 0x3FFFu);
+    uint32_t w[8];
+    if (kind == kFixed8) {
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(src) : "memory");
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(src + 16) : "memory");
+    } else {
+        uint4 c;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(c.x), "=r"(c.y), "=r"(c.z), "=r"(c.w) : "r"(src) : "memory");
+        if (kind == kPoT4) expand_pot_chunk(c, w); else expand_fixed4_chunk_x16(c, w);
     }
-}
-
-__device__ __forceinline__ void exp_store(const RawBuf& r, uint32_t a_stage, int q)
-{
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        const int kind = (r.meta[j] >> 8) & 3;
-        if (kind == 3) continue;
-        const int row = r.meta[j] & 0xFF;
-        uint32_t w[8];
-        if (kind == kFixed8) {
-            w[0] = r.lo[j].x; w[1] = r.lo[j].y; w[2] = r.lo[j].z; w[3] = r.lo[j].w;
-            w[4] = r.hi[j].x; w[5] = r.hi[j].y; w[6] = r.hi[j].z; w[7] = r.hi[j].w;
-        } else if (kind == kPoT4) {
-            expand_pot_chunk(r.lo[j], w);
-        } else {
-            expand_fixed4_chunk_x16(r.lo[j], w);
-        }
-        const uint32_t base = a_stage + row * 128;
-        const uint32_t sw = row & 7;
-        const uint32_t a0 = base + (((2 * q) ^ sw) << 4), a1 = base + (((2 * q + 1) ^ sw) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-    }
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst ^ 16u), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
 
 // ------------------------------------------------------------------ the kernel
 
 __global__ void __launch_bounds__(kThreads, 1)
-tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUtensorMap act_map,
-              const __grid_constant__ StoreMaps smaps)
+tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps maps)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sA = smem_base;
-    const uint32_t sB = smem_base + kStages * kABytes;
-    const uint32_t sOut = sB + kStages * kBBytes;
-    const uint32_t sBar = sOut + kStageOut;
-    // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]
-    const uint32_t bar_full = sBar, bar_empty = sBar + 8 * kStages;
-    const uint32_t bar_tfull = sBar + 16 * kStages, bar_tempty = bar_tfull + 16;
+    const uint32_t sB = sA + cfg.nA * kABytes;
+    const uint32_t sRaw = sB + cfg.nB * kBBytes;
+    const uint32_t sOut = sRaw + cfg.nR * cfg.raw_bytes;
+    const uint32_t sBar = sOut + kNumEpiWarps * cfg.out_bufs * kWarpStage;
+    // barriers, 8 bytes each
+    const uint32_t bar_fullA = sBar, bar_emptyA = sBar + 8 * kMaxRing;
+    const uint32_t bar_fullB = sBar + 16 * kMaxRing, bar_emptyB = sBar + 24 * kMaxRing;
+    const uint32_t bar_fullR = sBar + 32 * kMaxRing, bar_emptyR = sBar + 40 * kMaxRing;
+    const uint32_t bar_tfull = sBar + 48 * kMaxRing, bar_tempty = bar_tfull + 16;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar_full + 8 * s, 1 + kNumExpWarps);   // TMA producer + one arrival per expander warp
-            mbar_init(bar_empty + 8 * s, 1);                  // tcgen05.commit
+        for (int s = 0; s < kMaxRing; ++s) {
+            mbar_init(bar_fullA + 8 * s, 4);     // the four warps of one expander group
+            mbar_init(bar_emptyA + 8 * s, 1);    // tcgen05.commit
+            mbar_init(bar_fullB + 8 * s, 1);     // producer (+ transaction bytes)
+            mbar_init(bar_emptyB + 8 * s, 1);    // tcgen05.commit
+            mbar_init(bar_fullR + 8 * s, 1);     // producer (+ transaction bytes)
+            mbar_init(bar_emptyR + 8 * s, 4);    // the four warps of one expander group
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_tfull + 8 * b, 1);                  // tcgen05.commit
@@ -292,28 +310,58 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
     volatile int* abort_flag = &s_abort;
 
     const int64_t first = blockIdx.x, step = gridDim.x;
-    const int taps_w = p.kw;
+    const int64_t my_tiles = (cfg.ntiles > first) ? (cfg.ntiles - first + step - 1) / step : 0;
 
     if (warp == 0) {
         // ---------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            uint32_t g = 0;
-            for (int64_t tile = first; tile < cfg.ntiles && !*abort_flag; tile += step) {
+        // The whole warp takes part: lane 0 waits on the barriers and fetches the activation box,
+        // the weight boxes of a k-block are issued by one lane each.
+        {
+            uint32_t sb = 0, phB = 0, sr = 0, phR = 0;
+            bool ok = true;
+            for (int64_t tile = first; tile < cfg.ntiles && ok; tile += step) {
+                const int blk = (int)(tile % p.nblocks);
                 const int64_t nt = tile / p.nblocks;
                 int b0, h0;
                 if (cfg.tiles_per_image) { b0 = (int)(nt / cfg.tiles_per_image); h0 = (int)(nt % cfg.tiles_per_image) * cfg.th; }
                 else { b0 = (int)(nt * cfg.tb); h0 = 0; }
-                for (int kb = 0; kb < cfg.nkb; ++kb, ++g) {
-                    const int s = g % kStages;
-                    if (!mbar_wait(bar_empty + 8 * s, ((g / kStages) & 1) ^ 1, abort_flag)) break;
-                    const int tap = kb / cfg.cpt, c0 = (kb - tap * cfg.cpt) * 128;
-                    const int ti = tap / taps_w, tj = tap - ti * taps_w;
-                    mbar_arrive_expect_tx(bar_full + 8 * s, cfg.tx_bytes);
-                    tma_load_4d(sB + s * kBBytes, &act_map, bar_full + 8 * s, c0, tj - p.pad,
-                                h0 * p.stride + ti - p.pad, b0);
+                const BlockInfo bi = load_block(p, blk);
+                const int nbP = ceil_box(bi.nP) / kRawBoxRows, nbF = ceil_box(bi.nF) / kRawBoxRows,
+                          nbE = ceil_box(bi.nE) / kRawBoxRows;
+                const uint32_t raw_tx = (uint32_t)(nbP + nbF) * (kRawBoxRows * 64) + (uint32_t)nbE * (kRawBoxRows * 128);
+                // this lane's weight box (lanes beyond the box count have none)
+                const CUtensorMap* my_map = nullptr;
+                int my_row = 0, my_x8 = 0;           // my_x8: 1 if the box is in the 8-bit region
+                uint32_t my_dst = 0;
+                if (lane < nbP) { my_map = &maps.q4; my_row = bi.p0 + lane * kRawBoxRows; my_dst = lane * (kRawBoxRows * 64); }
+                else if (lane < nbP + nbF) { my_map = &maps.q4; my_row = p.nP + bi.f0 + (lane - nbP) * kRawBoxRows; my_dst = lane * (kRawBoxRows * 64); }
+                else if (lane < nbP + nbF + nbE) {
+                    my_map = &maps.q8; my_x8 = 1; my_row = bi.e0 + (lane - nbP - nbF) * kRawBoxRows;
+                    my_dst = (nbP + nbF) * (kRawBoxRows * 64) + (lane - nbP - nbF) * (kRawBoxRows * 128);
+                }
+                int tap = 0, cc = 0;
+                for (int kb = 0; kb < cfg.nkb; ++kb) {
+                    const int c0 = cc * 128, koff = tap * p.Cp + c0;
+                    // packed weights of this tile's rows, group by group
+                    if (!mbar_wait_warp(bar_emptyR + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t rbar = bar_fullR + 8 * sr;
+                    if (lane == 0) mbar_arrive_expect_tx(rbar, raw_tx);
+                    __syncwarp();
+                    if (my_map) tma_load_2d(sRaw + sr * cfg.raw_bytes + my_dst, my_map, rbar, my_x8 ? koff : (koff >> 1), my_row);
+                    if (++sr == (uint32_t)cfg.nR) { sr = 0; phR ^= 1; }
+                    // activation codes
+                    if (!mbar_wait_warp(bar_emptyB + 8 * sb, phB ^ 1, abort_flag)) { ok = false; break; }
+                    if (lane == 0) {
+                        const int ti = tap / p.kw, tj = tap - ti * p.kw;
+                        mbar_arrive_expect_tx(bar_fullB + 8 * sb, cfg.tx_bytes);
+                        tma_load_4d(sB + sb * kBBytes, &maps.act, bar_fullB + 8 * sb, c0, tj - p.pad,
+                                    h0 * p.stride + ti - p.pad, b0);
+                    }
+                    if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; }
+                    if (++cc == cfg.cpt) { cc = 0; ++tap; }
                 }
             }
-            if (*abort_flag) {
+            if (!ok && lane == 0) {
                 // give copies already in flight time to land before the CTA's memory is released
                 for (int i = 0; i < 200; ++i) __nanosleep(1000);
             }
@@ -321,23 +369,27 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
     } else if (warp == 1) {
         // ---------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            uint32_t g = 0, it = 0;
+            uint32_t sa = 0, phA = 0, sb = 0, phB = 0, it = 0;
             for (int64_t tile = first; tile < cfg.ntiles && !*abort_flag; tile += step, ++it) {
                 const uint32_t ab = it & 1;
                 if (!mbar_wait(bar_tempty + 8 * ab, ((it >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + ab * kTileN;
                 bool ok = true;
-                for (int kb = 0; kb < cfg.nkb; ++kb, ++g) {
-                    const int s = g % kStages;
-                    if (!mbar_wait(bar_full + 8 * s, (g / kStages) & 1, abort_flag)) { ok = false; break; }
+                int cc = 0;
+                for (int kb = 0; kb < cfg.nkb; ++kb) {
+                    if (!mbar_wait(bar_fullB + 8 * sb, phB, abort_flag) ||
+                        !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const int c0 = (kb % cfg.cpt) * 128;
-                    const int ksteps = (min(128, p.Cin - c0) + 31) >> 5;
-                    const uint64_t ad = smem_desc_sw128(sA + s * kABytes), bd = smem_desc_sw128(sB + s * kBBytes);
+                    const int ksteps = (cc == cfg.cpt - 1) ? cfg.last_ksteps : 4;
+                    const uint64_t ad = smem_desc_sw128(sA + sa * kABytes), bd = smem_desc_sw128(sB + sb * kBBytes);
                     for (int ks = 0; ks < ksteps; ++ks)
                         mma_i8(d_tmem, ad + 2 * ks, bd + 2 * ks, cfg.idesc, (kb | ks) ? 1u : 0u);
-                    mma_commit(bar_empty + 8 * s);
+                    mma_commit(bar_emptyA + 8 * sa);
+                    mma_commit(bar_emptyB + 8 * sb);
+                    if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; }
+                    if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; }
+                    if (++cc == cfg.cpt) cc = 0;
                 }
                 if (!ok) break;
                 mma_commit(bar_tfull + 8 * ab);
@@ -345,62 +397,69 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
         }
     } else if (warp < 2 + kNumExpWarps) {
         // ---------------------------------------------------------- expanders
-        const int et = threadIdx.x - 64;          // 0..255
-        const int q = et & 3;                     // k-step (32 codes) handled within each k-block
-        const int slot0 = et >> 2;                // rows slot0 and slot0 + 64 of the tile's sorted order
-        RowTask cur[2], nxt[2];
-        int64_t load_tile = first;                // tile the load cursor is in
-        cur[0] = make_task(p, load_tile < cfg.ntiles ? load_tile : -1, slot0);
-        cur[1] = make_task(p, load_tile < cfg.ntiles ? load_tile : -1, slot0 + 64);
-        {
-            const int64_t t2 = load_tile + step;
-            nxt[0] = make_task(p, t2 < cfg.ntiles ? t2 : -1, slot0);
-            nxt[1] = make_task(p, t2 < cfg.ntiles ? t2 : -1, slot0 + 64);
-        }
-        int load_kb = 0;
-        // k-blocks left for this CTA
-        int64_t my_tiles = (cfg.ntiles > first) ? (cfg.ntiles - first + step - 1) / step : 0;
+        const int grp = (warp - 2) >> 2;                 // which k-blocks: g % kGroups == grp
+        const int et = ((warp - 2) & 3) * 32 + lane;     // 0..127 inside the group
+        const int q = et & 3;                            // 32-code step inside each k-block
+        const int slot0 = et >> 2;                       // rows slot0 + 32*i of the tile's sorted order
+        // tile look-ahead: one tile, or kGroups tiles when every tile is a single k-block
+        const int64_t look = (cfg.nkb == 1) ? kGroups : 1;
         const int64_t total = my_tiles * cfg.nkb;
-
-        auto issue_load = [&](RawBuf& r, int64_t gl) {
-            // load cursor -> registers, then advance the cursor
-            if (gl >= total) { r.meta[0] = r.meta[1] = 3 << 8; return; }
-            const int tap = load_kb / cfg.cpt, c0 = (load_kb - tap * cfg.cpt) * 128;
-            const int ksteps = (min(128, p.Cin - c0) + 31) >> 5;
-            exp_load(r, cur, tap * p.Cp + c0 + q * 32, q < ksteps);
-            if (++load_kb == cfg.nkb) {
-                load_kb = 0;
-                load_tile += step;
-                cur[0] = nxt[0]; cur[1] = nxt[1];
-                const int64_t t2 = load_tile + step;
-                nxt[0] = make_task(p, t2 < cfg.ntiles ? t2 : -1, slot0);
-                nxt[1] = make_task(p, t2 < cfg.ntiles ? t2 : -1, slot0 + 64);
+        int64_t g = grp;                                 // this CTA's k-block counter
+        int64_t tl = g / cfg.nkb;                        // local tile index of g
+        int kb = (int)(g - tl * cfg.nkb);
+        int cc = kb % cfg.cpt;
+        uint32_t sa = (uint32_t)(g % cfg.nA), phA = (uint32_t)((g / cfg.nA) & 1);
+        uint32_t sr = (uint32_t)(g % cfg.nR), phR = (uint32_t)((g / cfg.nR) & 1);
+        uint32_t cur[4], nxt[4];
+        auto tile_of = [&](int64_t local) -> int64_t { return local < my_tiles ? first + local * step : -1; };
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            cur[i] = make_meta(p, tile_of(tl), slot0 + 32 * i, q);
+            nxt[i] = make_meta(p, tile_of(tl + look), slot0 + 32 * i, q);
+        }
+        while (g < total) {
+            const int ksteps = (cc == cfg.cpt - 1) ? cfg.last_ksteps : 4;
+            if (!mbar_wait_warp(bar_fullR + 8 * sr, phR, abort_flag)) break;
+            if (!mbar_wait_warp(bar_emptyA + 8 * sa, phA ^ 1, abort_flag)) break;
+            if (q < ksteps) {
+                const uint32_t rs = sRaw + sr * cfg.raw_bytes, as = sA + sa * kABytes;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if ((cur[i] >> 30) != 3u) expand_task(cur[i], rs, as);
             }
-        };
-        bool alive = true;
-        auto consume = [&](const RawBuf& r, int64_t g) {
-            const int s = (int)(g % kStages);
-            if (!mbar_wait_warp(bar_empty + 8 * s, (uint32_t)((g / kStages) & 1) ^ 1u, abort_flag)) { alive = false; return; }
-            exp_store(r, sA + s * kABytes, q);
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_full + 8 * s);
-        };
-
-        RawBuf r0, r1, r2;
-        issue_load(r0, 0);
-        issue_load(r1, 1);
-        for (int64_t g = 0; g < total && alive; g += 3) {
-            issue_load(r2, g + 2);
-            consume(r0, g);
-            if (g + 1 < total) { issue_load(r0, g + 3); consume(r1, g + 1); }
-            if (g + 2 < total) { issue_load(r1, g + 4); consume(r2, g + 2); }
+            if (lane == 0) {
+                mbar_arrive(bar_fullA + 8 * sa);
+                mbar_arrive(bar_emptyR + 8 * sr);
+            }
+            // advance by kGroups k-blocks
+            g += kGroups;
+            sa += kGroups; while (sa >= (uint32_t)cfg.nA) { sa -= cfg.nA; phA ^= 1; }
+            sr += kGroups; while (sr >= (uint32_t)cfg.nR) { sr -= cfg.nR; phR ^= 1; }
+            kb += kGroups;
+            cc += kGroups; while (cc >= cfg.cpt) cc -= cfg.cpt;
+            if (kb >= cfg.nkb) {
+                int64_t adv = 0;
+                while (kb >= cfg.nkb) { kb -= cfg.nkb; ++adv; }
+                tl += adv;
+                cc = kb % cfg.cpt;
+                if (adv == look) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) cur[i] = make_meta(p, tile_of(tl), slot0 + 32 * i, q);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) nxt[i] = make_meta(p, tile_of(tl + look), slot0 + 32 * i, q);
+            }
         }
     } else {
         // ---------------------------------------------------------- epilogue
         const int quarter = warp & 3;              // TMEM lanes this warp may read
-        const int half = (warp - (2 + kNumExpWarps)) >> 2;   // which chunks of a tile: even or odd
-        uint32_t it = 0;
+        const uint32_t my_stage = sOut + (uint32_t)(warp - (2 + kNumExpWarps)) * (cfg.out_bufs * kWarpStage);
+        uint32_t it = 0, stg_count = 0;
         for (int64_t tile = first; tile < cfg.ntiles; tile += step, ++it) {
             const uint32_t ab = it & 1;
             const int blk = (int)(tile % p.nblocks);
@@ -420,35 +479,30 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
             if (!mbar_wait_warp(bar_tfull + 8 * ab, (it >> 1) & 1, abort_flag)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * kTileN;
-            if (cfg.tma_store) {
-                // The warps of a tensor-memory quarter take alternate 32-pixel chunks of its 32 rows; each
-                // stages its chunk in a private buffer and issues its own bulk store, so no epilogue
-                // warp ever waits for another.
-                if (blk * kBlockRows + quarter * 32 >= p.M) {      // no valid row in this quarter
-                    tc_fence_before();
-                    if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
-                    continue;
-                }
-                const uint32_t stg = sOut + (uint32_t)(warp - (2 + kNumExpWarps)) * kWarpStage;
-                const int nchunks = (nvalid + 31) >> 5;
-                if (half >= nchunks) {                             // a one-chunk tile leaves the odd warps idle
-                    tc_fence_before();
-                    if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
-                    continue;
-                }
-                for (int c = half; c < nchunks; c += kEpiPerQuarter) {
-                    uint32_t v[32];
-                    tmem_ld32(taddr + c * 32, v);
-                    if (c + kEpiPerQuarter >= nchunks) {
-                        // all accumulators of this tile are in registers: hand the buffer back
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
-                    }
+            const int nchunks = (nvalid + 31) >> 5;
+            auto release_tmem = [&]() {
+                // all accumulators of this tile are in registers: hand the buffer back
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
+            };
+            if (blk * kBlockRows + quarter * 32 >= p.M) {      // no valid row in this quarter
+                release_tmem();
+                continue;
+            }
+            // Output one 32-pixel chunk held in registers.
+            auto emit = [&](const uint32_t (&v)[32], int c) {
+                const int jmax = min(32, nvalid - c * 32);
+                if (cfg.tma_store) {
                     const bool tail = cfg.tail_rows && (c == (cfg.npix >> 5));
                     const int nsub = p.acc ? 2 : 1;
                     for (int sub = 0; sub < nsub; ++sub) {
-                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        const uint32_t stg = my_stage + (cfg.out_bufs == 2 ? (stg_count & 1) * kWarpStage : 0);
+                        ++stg_count;
+                        if (lane == 0) {
+                            if (cfg.out_bufs == 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                            else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        }
                         __syncwarp();                    // the buffer's previous store has been read out
                         if (!p.out_mn) {
                             // [pixel][row]: the warp writes 128 contiguous bytes per pixel
@@ -463,34 +517,28 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
                             // [row][pixel], 16-byte chunks swizzled by row (matches the 128-byte-swizzled store map)
                             const uint32_t a0 = stg + lane * 128;
 #pragma unroll
-                            for (int cc = 0; cc < 8; ++cc) {
+                            for (int cch = 0; cch < 8; ++cch) {
                                 uint32_t w[4];
 #pragma unroll
                                 for (int t = 0; t < 4; ++t) {
-                                    const int a = (int)v[4 * cc + t] >> shift;
+                                    const int a = (int)v[4 * cch + t] >> shift;
                                     w[t] = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
                                 }
                                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                                             ::"r"(a0 + ((cc ^ (lane & 7)) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+                                             ::"r"(a0 + ((cch ^ (lane & 7)) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
                             }
                         }
                         fence_proxy_async_smem();
                         __syncwarp();                    // chunk complete in shared memory
                         if (lane == 0) {
-                            const CUtensorMap* map = sub ? (tail ? &smaps.acc_tail : &smaps.acc_full)
-                                                         : (tail ? &smaps.out_tail : &smaps.out_full);
+                            const CUtensorMap* map = sub ? (tail ? &maps.acc_tail : &maps.acc_full)
+                                                         : (tail ? &maps.out_tail : &maps.out_full);
                             const int cm = blk * kBlockRows + quarter * 32, cn = (int)(n0 + c * 32);
                             if (!p.out_mn) tma_store_2d(map, stg, cm, cn); else tma_store_2d(map, stg, cn, cm);
                         }
                     }
-                }
-                continue;
-            }
-            for (int c = 0; c * 32 < nvalid; ++c) {
-                uint32_t v[32];
-                tmem_ld32(taddr + c * 32, v);
-                const int jmax = min(32, nvalid - c * 32);
-                if (row_ok) {
+                } else if (row_ok) {
+                    // direct stores: outputs whose leading dimension or base rules out bulk stores
                     if (!p.out_mn) {
                         float* o = p.out + (n0 + c * 32) * p.ld_out + m;
                         int32_t* oa = p.acc ? p.acc + (n0 + c * 32) * p.ld_out + m : nullptr;
@@ -505,40 +553,38 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ CUte
                     } else {
                         float* o = p.out + (int64_t)m * p.ld_out + n0 + c * 32;
                         int32_t* oa = p.acc ? p.acc + (int64_t)m * p.ld_out + n0 + c * 32 : nullptr;
-                        const bool vec = (jmax == 32) && ((reinterpret_cast<uintptr_t>(o) & 15) == 0);
-                        if (vec) {
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                float4 f;
-                                f.x = __fmul_rn(__int2float_rn((int)v[j] >> shift), scale);
-                                f.y = __fmul_rn(__int2float_rn((int)v[j + 1] >> shift), scale);
-                                f.z = __fmul_rn(__int2float_rn((int)v[j + 2] >> shift), scale);
-                                f.w = __fmul_rn(__int2float_rn((int)v[j + 3] >> shift), scale);
-                                *reinterpret_cast<float4*>(o + j) = f;
-                                if (oa) *reinterpret_cast<int4*>(oa + j) = make_int4((int)v[j] >> shift, (int)v[j + 1] >> shift,
-                                                                                     (int)v[j + 2] >> shift, (int)v[j + 3] >> shift);
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                if (j < jmax) {
-                                    const int a = (int)v[j] >> shift;
-                                    o[j] = __fmul_rn(__int2float_rn(a), scale);
-                                    if (oa) oa[j] = a;
-                                }
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < jmax) {
+                                const int a = (int)v[j] >> shift;
+                                o[j] = __fmul_rn(__int2float_rn(a), scale);
+                                if (oa) oa[j] = a;
                             }
                         }
                     }
                 }
+            };
+            // two register sets: the load of chunk c+1 is in flight while chunk c is emitted
+            uint32_t va[32], vb[32];
+            tmem_ld_issue(taddr, va);
+            tmem_ld_wait(va);
+            for (int c = 0; c < nchunks; c += 2) {
+                const bool more1 = c + 1 < nchunks;
+                if (more1) tmem_ld_issue(taddr + (c + 1) * 32, vb); else release_tmem();
+                emit(va, c);
+                if (more1) {
+                    tmem_ld_wait(vb);
+                    const bool more2 = c + 2 < nchunks;
+                    if (more2) tmem_ld_issue(taddr + (c + 2) * 32, va); else release_tmem();
+                    emit(vb, c + 1);
+                    if (more2) tmem_ld_wait(va);
+                }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     // ---------------------------------------------------------- teardown
-    if (warp >= 2 + kNumExpWarps && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -576,6 +622,7 @@ bool plan(const Problem& p, TensorCfg& c)
 {
     if (p.pix_pitch % 16 != 0 || p.Cin % 16 != 0) return false;
     if ((reinterpret_cast<uintptr_t>(p.act) & 15) != 0) return false;
+    if (p.raw_stage_bytes <= 0) return false;
     const int64_t hw = (int64_t)p.Ho * p.Wo;
     if (p.Wo > kTileN || (int64_t)p.Wo * p.stride > 256) return false;
     if (hw <= kTileN) {
@@ -597,11 +644,27 @@ bool plan(const Problem& p, TensorCfg& c)
     c.ntiles = c.ntiles_n * p.nblocks;
     c.cpt = (p.Cin + 127) / 128;
     c.nkb = p.kh * p.kw * c.cpt;
+    c.last_ksteps = (p.Cin - (c.cpt - 1) * 128 + 31) / 32;
     c.tx_bytes = (uint32_t)c.npix * 128u;
     // kind::i8: int32 accumulate (bits 4-5 = 2), signed 8-bit A and B (bits 7-9, 10-12 = 1),
     // both K-major, N/8 at bit 17, M/16 at bit 24
     c.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.n_mma >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
-    return true;
+    c.tail_rows = c.npix & 31;
+    c.tma_store = 0;
+    // shared-memory budget: rings as deep as fit
+    c.raw_bytes = ((uint32_t)p.raw_stage_bytes + 1023u) & ~1023u;
+    const int fixed = 1024 /*alignment*/ + 64 * kMaxRing /*barriers*/;
+    struct Choice { int nA, nB, nR, ob; };
+    const Choice order[] = {{3, 4, 3, 2}, {3, 4, 3, 1}, {3, 3, 3, 2}, {2, 3, 3, 2}, {2, 3, 2, 1}, {2, 2, 2, 1}};
+    for (const Choice& ch : order) {
+        const int64_t need = (int64_t)ch.nA * kABytes + (int64_t)ch.nB * kBBytes + (int64_t)ch.nR * c.raw_bytes +
+                             (int64_t)kNumEpiWarps * ch.ob * kWarpStage + fixed;
+        if (need <= kSmemLimit) {
+            c.nA = ch.nA; c.nB = ch.nB; c.nR = ch.nR; c.out_bufs = ch.ob; c.smem_bytes = (uint32_t)need;
+            return true;
+        }
+    }
+    return false;
 }
 
 }  // namespace
@@ -618,44 +681,54 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
     if (!plan(p, c)) return RMSMP_ERR_VARIANT;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return RMSMP_ERR_CUDA;
-    CUtensorMap map;
-    const cuuint64_t gdim[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
-    const cuuint64_t gstr[3] = {(cuuint64_t)p.pix_pitch, (cuuint64_t)p.pix_pitch * p.W,
-                                (cuuint64_t)p.pix_pitch * p.W * p.H};
-    const cuuint32_t box[4] = {128u, (cuuint32_t)(p.Wo * p.stride), (cuuint32_t)(c.th * p.stride), (cuuint32_t)c.tb};
-    const cuuint32_t estr[4] = {1u, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1u};
-    CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(p.act), gdim, gstr, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return RMSMP_ERR_CUDA;
+    Maps mp;
+    memset(&mp, 0, sizeof(mp));
+    {
+        const cuuint64_t gdim[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+        const cuuint64_t gstr[3] = {(cuuint64_t)p.pix_pitch, (cuuint64_t)p.pix_pitch * p.W,
+                                    (cuuint64_t)p.pix_pitch * p.W * p.H};
+        const cuuint32_t box[4] = {128u, (cuuint32_t)(p.Wo * p.stride), (cuuint32_t)(c.th * p.stride), (cuuint32_t)c.tb};
+        const cuuint32_t estr[4] = {1u, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1u};
+        if (enc(&mp.act, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(p.act), gdim, gstr, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return RMSMP_ERR_CUDA;
+    }
+    // packed weight regions: rows of Kp/2 (4-bit) and Kp (8-bit) bytes, boxes of 16 rows x one k-block
+    auto make_w = [&](CUtensorMap* m, const uint8_t* base, int rows, int pitch, int box_bytes) -> bool {
+        if (rows <= 0) return true;
+        const cuuint64_t gd[2] = {(cuuint64_t)pitch, (cuuint64_t)rows};
+        const cuuint64_t gs[1] = {(cuuint64_t)pitch};
+        const cuuint32_t bx[2] = {(cuuint32_t)box_bytes, (cuuint32_t)kRawBoxRows};
+        const cuuint32_t es[2] = {1, 1};
+        return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), gd, gs, bx, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    if (!make_w(&mp.q4, p.q4, p.nP + p.nF4, p.Kp / 2, 64) || !make_w(&mp.q8, p.q8, p.n8, p.Kp, 128))
+        return RMSMP_ERR_CUDA;
 
-    StoreMaps sm;
-    memset(&sm, 0, sizeof(sm));
-    c.tma_store = 0;
-    c.tail_rows = c.npix & 31;
     const bool ld_ok = (p.ld_out % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
                        (!p.acc || (reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
     if (ld_ok && (!p.out_mn || c.tail_rows == 0)) {
         auto make = [&](CUtensorMap* m, void* base, CUtensorMapDataType dt, int rows) -> bool {
+            const cuuint32_t es[2] = {1, 1};
+            const cuuint64_t gs[1] = {(cuuint64_t)p.ld_out * 4};
             if (!p.out_mn) {
                 const cuuint64_t gd[2] = {(cuuint64_t)p.M, (cuuint64_t)p.N};
-                const cuuint64_t gs[1] = {(cuuint64_t)p.ld_out * 4};
                 const cuuint32_t bx[2] = {32u, (cuuint32_t)rows};
-                const cuuint32_t es[2] = {1, 1};
                 return enc(m, dt, 2, base, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
             }
             const cuuint64_t gd[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
-            const cuuint64_t gs[1] = {(cuuint64_t)p.ld_out * 4};
             const cuuint32_t bx[2] = {32u, 32u};
-            const cuuint32_t es[2] = {1, 1};
             return enc(m, dt, 2, base, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                        CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
         };
-        bool ok = make(&sm.out_full, p.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 32);
-        if (ok && c.tail_rows) ok = make(&sm.out_tail, p.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.tail_rows);
-        if (ok && p.acc) ok = make(&sm.acc_full, p.acc, CU_TENSOR_MAP_DATA_TYPE_INT32, 32);
-        if (ok && p.acc && c.tail_rows) ok = make(&sm.acc_tail, p.acc, CU_TENSOR_MAP_DATA_TYPE_INT32, c.tail_rows);
+        bool ok = make(&mp.out_full, p.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 32);
+        if (ok && c.tail_rows) ok = make(&mp.out_tail, p.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.tail_rows);
+        if (ok && p.acc) ok = make(&mp.acc_full, p.acc, CU_TENSOR_MAP_DATA_TYPE_INT32, 32);
+        if (ok && p.acc && c.tail_rows) ok = make(&mp.acc_tail, p.acc, CU_TENSOR_MAP_DATA_TYPE_INT32, c.tail_rows);
         c.tma_store = ok ? 1 : 0;
     }
 
@@ -665,14 +738,14 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (cudaFuncSetAttribute(tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
             cudaGetLastError();
             return RMSMP_ERR_CUDA;
         }
         attr_set = true;
     }
     const int grid = (int)std::min<int64_t>(c.ntiles, sm_count > 0 ? sm_count : 148);
-    tensor_kernel<<<grid, kThreads, kSmemBytes, st>>>(p, c, map, sm);
+    tensor_kernel<<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
     if (cudaGetLastError() != cudaSuccess) return RMSMP_ERR_CUDA;
     return RMSMP_OK;
 }
