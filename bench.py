@@ -163,19 +163,31 @@ def run_ours(args):
         D.append(dict(
             W=torch.from_numpy(h["W"]).cuda(), x=torch.from_numpy(h["x"]).cuda(),
             packed=torch.empty(h["lay"].packed_bytes, dtype=torch.uint8, device="cuda"),
+            ws=torch.empty(R.rmsmp_workspace_bytes(h["lay"]), dtype=torch.int8, device="cuda"),
             codes=torch.empty(h["x"].shape, dtype=torch.int8, device="cuda"),
             y=torch.empty((N, L.M), dtype=torch.float32, device="cuda"), N=N))
 
+    use_ws = (args.variant == "workspace")
+
+    def conv(h, d, st):
+        L = h["L"]
+        if use_ws:
+            R.rmsmp_conv_implicit_workspace(h["lay"], d["packed"], d["ws"], d["codes"], batch, L.H, L.H, L.stride,
+                                            L.pad, st, d["y"], R.OUT_NM, None, stream=stream)
+        else:
+            R.rmsmp_conv_implicit_variant(h["lay"], d["packed"], d["codes"], batch, L.H, L.H, L.stride, L.pad, st,
+                                          d["y"], R.OUT_NM, None, R.VARIANT_TENSOR, stream=stream)
+
     def step(ev=None):
         for i, (h, d) in enumerate(zip(H, D)):
-            L = h["L"]
             R.rmsmp_quantize_pack(d["W"], R.W_CONV_OIHW, h["lay"], h["scheme"], h["bits"], h["alpha"],
                                   R.POT_NEAREST, d["packed"], stream=stream)
+            if use_ws:
+                R.rmsmp_expand_weights(h["lay"], d["packed"], d["ws"], stream=stream)
             st = R.rmsmp_quantize_act(d["x"], d["x"].numel(), synth.ALPHA_ACT, R.ACT_U4, d["codes"], stream=stream)
             if ev is not None:
                 ev[i][0].record(stream)
-            R.rmsmp_conv_implicit(h["lay"], d["packed"], d["codes"], batch, L.H, L.H, L.stride, L.pad, st,
-                                  d["y"], R.OUT_NM, None, stream=stream)
+            conv(h, d, st)
             if ev is not None:
                 ev[i][1].record(stream)
 
@@ -233,9 +245,10 @@ def run_ours(args):
             d["x"].copy_(p["x"], non_blocking=True)
             R.rmsmp_quantize_pack(d["W"], R.W_CONV_OIHW, h["lay"], h["scheme"], h["bits"], h["alpha"],
                                   R.POT_NEAREST, d["packed"], stream=stream)
+            if use_ws:
+                R.rmsmp_expand_weights(h["lay"], d["packed"], d["ws"], stream=stream)
             st = R.rmsmp_quantize_act(d["x"], d["x"].numel(), synth.ALPHA_ACT, R.ACT_U4, d["codes"], stream=stream)
-            R.rmsmp_conv_implicit(h["lay"], d["packed"], d["codes"], batch, L.H, L.H, L.stride, L.pad, st,
-                                  d["y"], R.OUT_NM, None, stream=stream)
+            conv(h, d, st)
             p["y"].copy_(d["y"], non_blocking=True)
 
     if e2e_steps:
@@ -268,11 +281,11 @@ def run_ours(args):
         "data": "synthetic",
         "config": {"workload": WORKLOAD if LAYER_FILTER is None else "subset:" + ",".join(sorted(LAYER_FILTER)), "batch_per_gpu": batch, "layers": len(layers),
                    "ops_per_step_per_gpu": ops_step, "l2": "inputs larger than L2 (every layer reads 13-205 MB and writes 6-205 MB)",
-                   "step": "per layer: quantize_pack + quantize_act + conv_implicit (tensor variant)"},
+                   "step": "per layer: quantize_pack%s + quantize_act + conv_implicit (tensor cores, %s)" % ((" + expand_weights", "weights expanded once into scratch") if use_ws else ("", "weights expanded in shared memory per tile"))},
         "clocks": clocks,
         "e2e": ({"value": world * ops_step / (e2e_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_step,
                  "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h} if e2e_steps else None),
-        "gpu_launches": args.steps * len(layers) * 3,
+        "gpu_launches": args.steps * len(layers) * (4 if use_ws else 3),
         "roofline": {"bound": "hbm", "kernel": "tensor_kernel (conv_implicit)", "achieved": achieved_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved_gbs / peaks["hbm_gbs"],
                      "peak_source": peak_src, "traffic": TRAFFIC_PER_STEP_BYTES,
@@ -373,6 +386,9 @@ def main():
     ap.add_argument("--cpu-sample-batch", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--variant", default="workspace", choices=["workspace", "smem"],
+                    help="tensor-core path: expand the weight codes once into scratch memory (default) "
+                         "or in shared memory per tile")
     ap.add_argument("--layers", default=None,
                     help="comma-separated layer names: run one instance of each (profiling runs)")
     args = ap.parse_args()

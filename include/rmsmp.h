@@ -200,6 +200,34 @@ rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* layer, const void* d
                                          rmsmp_variant variant, void* stream);
 
 /*
+ * Workspace variant of the tensor-core path.  The expansion of the 4-bit / PoT codes to int8
+ * (the GPU counterpart of routing rows to the per-scheme GEMM cores, Section 4.1) is done ONCE
+ * per layer into caller-provided scratch memory instead of once per output tile in shared
+ * memory; the contraction kernel then fetches plain int8 rows with TMA.  Same results bit for
+ * bit.  Worth it when N is large (the expansion is amortised over all pixels).
+ *   rmsmp_workspace_bytes   size of the scratch buffer for a layer (M * Kp bytes, rounded up).
+ *   rmsmp_expand_weights    fills d_workspace ([M][Kp] int8 values, original row order, packed
+ *                           reduction order) from the packed buffer; must be repeated whenever
+ *                           the packed buffer changes.  d_workspace: 16-byte aligned.
+ *   rmsmp_gemm_workspace / rmsmp_conv_implicit_workspace
+ *                           as rmsmp_gemm / rmsmp_conv_implicit, A operand read from d_workspace.
+ * Errors: as the plain calls, plus BUFFER_TOO_SMALL; VARIANT when the tensor kernel cannot run
+ * the problem (K or Cin not a multiple of 16, ...).
+ */
+rmsmp_status rmsmp_workspace_bytes(const rmsmp_layer* layer, size_t* bytes);
+rmsmp_status rmsmp_expand_weights(const rmsmp_layer* layer, const void* d_packed, void* d_workspace,
+                                  size_t workspace_bytes, void* stream);
+rmsmp_status rmsmp_gemm_workspace(const rmsmp_layer* layer, const void* d_packed,
+                                  const void* d_workspace, const int8_t* d_act, int64_t N,
+                                  int64_t ld_act, float act_step, float* d_out, int64_t ld_out,
+                                  rmsmp_out_layout out_layout, int32_t* d_acc, void* stream);
+rmsmp_status rmsmp_conv_implicit_workspace(const rmsmp_layer* layer, const void* d_packed,
+                                           const void* d_workspace, const int8_t* d_act, int B,
+                                           int H, int W, int stride, int pad, float act_step,
+                                           float* d_out, rmsmp_out_layout out_layout,
+                                           int32_t* d_acc, void* stream);
+
+/*
  * Read the device status word of a packed buffer (synchronises the stream).  Kernels never
  * trap: a bounded wait that runs out stores RMSMP_ERR_TIMEOUT there and the kernel returns.
  */

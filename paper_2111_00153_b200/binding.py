@@ -29,7 +29,8 @@ EXPORTS = (
     "rmsmp_status_string", "rmsmp_assign_rows", "rmsmp_layer_init", "rmsmp_quantize_pack",
     "rmsmp_unpack_codes", "rmsmp_quantize_act", "rmsmp_gemm", "rmsmp_gemm_variant",
     "rmsmp_conv_implicit", "rmsmp_conv_implicit_variant", "rmsmp_last_device_status",
-    "rmsmp_measure_mma_peak",
+    "rmsmp_measure_mma_peak", "rmsmp_workspace_bytes", "rmsmp_expand_weights", "rmsmp_gemm_workspace",
+    "rmsmp_conv_implicit_workspace",
 )
 
 
@@ -90,6 +91,11 @@ def lib() -> C.CDLL:
         L.rmsmp_conv_implicit_variant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i32, i32, i32,
                                                   i32, i32, f32, vp, i32, vp, i32, vp]
         L.rmsmp_last_device_status.argtypes = [vp, vp]
+        L.rmsmp_workspace_bytes.argtypes = [C.POINTER(rmsmp_layer), C.POINTER(C.c_size_t)]
+        L.rmsmp_expand_weights.argtypes = [C.POINTER(rmsmp_layer), vp, vp, C.c_size_t, vp]
+        L.rmsmp_gemm_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
+        L.rmsmp_conv_implicit_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
+                                                    f32, vp, i32, vp, vp]
         L.rmsmp_measure_mma_peak.argtypes = [i32, i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
         _lib = L
     return _lib
@@ -204,6 +210,34 @@ def rmsmp_conv_implicit_variant(layer, d_packed, d_act, B: int, H: int, W: int, 
                                              stride, pad, act_step, _dp(d_out), out_layout,
                                              _dp(d_acc), variant, _stream(stream)),
            "rmsmp_conv_implicit_variant")
+
+
+def rmsmp_workspace_bytes(layer) -> int:
+    n = C.c_size_t(0)
+    _check(lib().rmsmp_workspace_bytes(C.byref(layer), C.byref(n)), "rmsmp_workspace_bytes")
+    return n.value
+
+
+def rmsmp_expand_weights(layer, d_packed, d_workspace, workspace_bytes: int | None = None, stream=None):
+    if workspace_bytes is None:
+        workspace_bytes = d_workspace.numel() * d_workspace.element_size()
+    _check(lib().rmsmp_expand_weights(C.byref(layer), _dp(d_packed), _dp(d_workspace), workspace_bytes,
+                                      _stream(stream)), "rmsmp_expand_weights")
+
+
+def rmsmp_gemm_workspace(layer, d_packed, d_workspace, d_act, N: int, ld_act: int, act_step: float,
+                         d_out, ld_out: int, out_layout: int = OUT_NM, d_acc=None, stream=None):
+    _check(lib().rmsmp_gemm_workspace(C.byref(layer), _dp(d_packed), _dp(d_workspace), _dp(d_act), N,
+                                      ld_act, act_step, _dp(d_out), ld_out, out_layout, _dp(d_acc),
+                                      _stream(stream)), "rmsmp_gemm_workspace")
+
+
+def rmsmp_conv_implicit_workspace(layer, d_packed, d_workspace, d_act, B: int, H: int, W: int,
+                                  stride: int, pad: int, act_step: float, d_out,
+                                  out_layout: int = OUT_NM, d_acc=None, stream=None):
+    _check(lib().rmsmp_conv_implicit_workspace(C.byref(layer), _dp(d_packed), _dp(d_workspace), _dp(d_act),
+                                               B, H, W, stride, pad, act_step, _dp(d_out), out_layout,
+                                               _dp(d_acc), _stream(stream)), "rmsmp_conv_implicit_workspace")
 
 
 def rmsmp_last_device_status(d_packed, stream=None) -> int:

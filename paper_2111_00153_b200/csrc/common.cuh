@@ -35,6 +35,7 @@ struct Problem {
     const int32_t* blocks;    // [nblocks][8]
     const uint8_t* q4;        // [(nP+nF4)][Kp/2]
     const uint8_t* q8;        // [n8][Kp]
+    const int8_t* wexp;       // [M][Kp] int8 values in original row order, or null (workspace variant)
     uint32_t* status;
     int M, Cin, kh, kw, Cp, Kp, nP, nF4, n8, nblocks, raw_stage_bytes;
     // activations: [B][H][W] pixels of `pix_pitch` bytes, Cin codes used in each
@@ -55,6 +56,7 @@ cudaError_t launch_pack(const float* dW, int conv_oihw, const rmsmp_layer& L, in
                         uint8_t* blob, cudaStream_t st);
 cudaError_t launch_unpack(const rmsmp_layer& L, const uint8_t* blob, int8_t* values,
                           int32_t* perm, float* wstep, cudaStream_t st);
+cudaError_t launch_expand(const rmsmp_layer& L, const uint8_t* blob, int8_t* wexp, cudaStream_t st);
 cudaError_t launch_quantize_act(const float* x, size_t count, float alpha, int kind, int8_t* codes,
                                 cudaStream_t st);
 cudaError_t launch_simple(const Problem& p, cudaStream_t st);

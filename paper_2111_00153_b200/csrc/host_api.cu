@@ -61,6 +61,7 @@ void fill_problem(Problem& p, const rmsmp_layer* L, const void* d_packed)
     p.M = L->M; p.Cin = L->Cin; p.kh = L->kh; p.kw = L->kw; p.Cp = L->Cp; p.Kp = L->Kp;
     p.nP = L->nP; p.nF4 = L->nF4; p.n8 = L->n8; p.nblocks = L->nblocks;
     p.raw_stage_bytes = L->raw_stage_bytes;
+    p.wexp = nullptr;
 }
 
 rmsmp_status dispatch(Problem& p, rmsmp_variant variant, cudaStream_t st)
@@ -280,12 +281,12 @@ rmsmp_status rmsmp_quantize_act(const float* d_X, size_t count, float alpha_a, r
     return RMSMP_OK;
 }
 
-rmsmp_status rmsmp_gemm_variant(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act,
-                                int64_t N, int64_t ld_act, float act_step, float* d_out,
-                                int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
-                                rmsmp_variant variant, void* stream)
+static rmsmp_status gemm_impl(const rmsmp_layer* L, const void* d_packed, const void* d_ws, bool use_ws,
+                              const int8_t* d_act, int64_t N, int64_t ld_act, float act_step, float* d_out,
+                              int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
+                              rmsmp_variant variant, void* stream)
 {
-    if (!L || !d_packed || !d_act || !d_out) return RMSMP_ERR_NULL;
+    if (!L || !d_packed || !d_act || !d_out || (use_ws && !d_ws)) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     if (L->kh != 1 || L->kw != 1) return RMSMP_ERR_SHAPE;
     if (N < 1 || N > (int64_t)1 << 31 || ld_act < L->Cin) return RMSMP_ERR_SHAPE;
@@ -304,7 +305,29 @@ rmsmp_status rmsmp_gemm_variant(const rmsmp_layer* L, const void* d_packed, cons
     p.pix_pitch = ld_act; p.N = N;
     p.act_step = act_step; p.out = d_out; p.acc = d_acc; p.ld_out = ld_out;
     p.out_mn = (out_layout == RMSMP_OUT_MN);
+    if (use_ws) {
+        if (!aligned16(d_ws)) return RMSMP_ERR_ALIGN;
+        p.wexp = static_cast<const int8_t*>(d_ws);
+    }
     return dispatch(p, variant, static_cast<cudaStream_t>(stream));
+}
+
+rmsmp_status rmsmp_gemm_variant(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act,
+                                int64_t N, int64_t ld_act, float act_step, float* d_out,
+                                int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
+                                rmsmp_variant variant, void* stream)
+{
+    return gemm_impl(L, d_packed, nullptr, false, d_act, N, ld_act, act_step, d_out, ld_out, out_layout, d_acc,
+                     variant, stream);
+}
+
+rmsmp_status rmsmp_gemm_workspace(const rmsmp_layer* L, const void* d_packed, const void* d_workspace,
+                                  const int8_t* d_act, int64_t N, int64_t ld_act, float act_step,
+                                  float* d_out, int64_t ld_out, rmsmp_out_layout out_layout,
+                                  int32_t* d_acc, void* stream)
+{
+    return gemm_impl(L, d_packed, d_workspace, true, d_act, N, ld_act, act_step, d_out, ld_out, out_layout,
+                     d_acc, RMSMP_VARIANT_TENSOR, stream);
 }
 
 rmsmp_status rmsmp_gemm(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act, int64_t N,
@@ -315,13 +338,12 @@ rmsmp_status rmsmp_gemm(const rmsmp_layer* L, const void* d_packed, const int8_t
                               d_acc, RMSMP_VARIANT_AUTO, stream);
 }
 
-rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* L, const void* d_packed,
-                                         const int8_t* d_act, int B, int H, int W, int stride,
-                                         int pad, float act_step, float* d_out,
-                                         rmsmp_out_layout out_layout, int32_t* d_acc,
-                                         rmsmp_variant variant, void* stream)
+static rmsmp_status conv_impl(const rmsmp_layer* L, const void* d_packed, const void* d_ws, bool use_ws,
+                              const int8_t* d_act, int B, int H, int W, int stride, int pad, float act_step,
+                              float* d_out, rmsmp_out_layout out_layout, int32_t* d_acc,
+                              rmsmp_variant variant, void* stream)
 {
-    if (!L || !d_packed || !d_act || !d_out) return RMSMP_ERR_NULL;
+    if (!L || !d_packed || !d_act || !d_out || (use_ws && !d_ws)) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     if (B < 1 || H < 1 || W < 1 || stride < 1 || stride > 8 || pad < 0 || pad > 16) return RMSMP_ERR_SHAPE;
     if (H + 2 * pad < L->kh || W + 2 * pad < L->kw) return RMSMP_ERR_SHAPE;
@@ -343,7 +365,55 @@ rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* L, const void* d_pac
     p.act_step = act_step; p.out = d_out; p.acc = d_acc;
     p.out_mn = (out_layout == RMSMP_OUT_MN);
     p.ld_out = p.out_mn ? N : L->M;
+    if (use_ws) {
+        if (!aligned16(d_ws)) return RMSMP_ERR_ALIGN;
+        p.wexp = static_cast<const int8_t*>(d_ws);
+    }
     return dispatch(p, variant, static_cast<cudaStream_t>(stream));
+}
+
+rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* L, const void* d_packed,
+                                         const int8_t* d_act, int B, int H, int W, int stride,
+                                         int pad, float act_step, float* d_out,
+                                         rmsmp_out_layout out_layout, int32_t* d_acc,
+                                         rmsmp_variant variant, void* stream)
+{
+    return conv_impl(L, d_packed, nullptr, false, d_act, B, H, W, stride, pad, act_step, d_out, out_layout,
+                     d_acc, variant, stream);
+}
+
+rmsmp_status rmsmp_conv_implicit_workspace(const rmsmp_layer* L, const void* d_packed,
+                                           const void* d_workspace, const int8_t* d_act, int B, int H,
+                                           int W, int stride, int pad, float act_step, float* d_out,
+                                           rmsmp_out_layout out_layout, int32_t* d_acc, void* stream)
+{
+    return conv_impl(L, d_packed, d_workspace, true, d_act, B, H, W, stride, pad, act_step, d_out, out_layout,
+                     d_acc, RMSMP_VARIANT_TENSOR, stream);
+}
+
+rmsmp_status rmsmp_workspace_bytes(const rmsmp_layer* L, size_t* bytes)
+{
+    if (!L || !bytes) return RMSMP_ERR_NULL;
+    if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+    *bytes = (size_t)align_up((uint64_t)L->M * L->Kp, 256);
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_expand_weights(const rmsmp_layer* L, const void* d_packed, void* d_workspace,
+                                  size_t workspace_bytes, void* stream)
+{
+    if (!L || !d_packed || !d_workspace) return RMSMP_ERR_NULL;
+    if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+    if (workspace_bytes < (size_t)L->M * L->Kp) return RMSMP_ERR_BUFFER_TOO_SMALL;
+    if (!aligned16(d_workspace) || (reinterpret_cast<uintptr_t>(d_packed) & 255)) return RMSMP_ERR_ALIGN;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    if (launch_expand(*L, static_cast<const uint8_t*>(d_packed), static_cast<int8_t*>(d_workspace),
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return RMSMP_OK;
 }
 
 rmsmp_status rmsmp_conv_implicit(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act,

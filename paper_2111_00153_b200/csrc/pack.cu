@@ -1,5 +1,6 @@
 // Weight quantize + group + pack, its inverse (parity/debug), and the activation quantizer.
 #include "common.cuh"
+#include "decode.cuh"
 
 namespace rmsmp {
 
@@ -184,6 +185,58 @@ cudaError_t launch_unpack(const rmsmp_layer& L, const uint8_t* blob, int8_t* val
     int64_t total = (int64_t)L.M * L.Cin * L.kh * L.kw;
     int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     unpack_kernel<<<blocks, 256, 0, st>>>(blob, L, values, perm, wstep);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ expand to int8 (workspace variant)
+// One thread per 32 codes: a 128-bit load of packed 4-bit codes (or two of 8-bit codes) becomes two
+// 128-bit stores of exact int8 values, rows in ORIGINAL order, reduction index as in the packed rows.
+
+__global__ void __launch_bounds__(256) expand_kernel(const uint8_t* __restrict__ blob, rmsmp_layer L,
+                                                     int8_t* __restrict__ wexp)
+{
+    const int chunks = L.Kp >> 5;
+    const int64_t total = (int64_t)L.M * chunks;
+    const int32_t* slot = reinterpret_cast<const int32_t*>(blob + L.off_slot);
+    const uint8_t* kind = blob + L.off_kind;
+    const int n4 = L.nP + L.nF4;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int m = (int)(i / chunks), c = (int)(i % chunks);
+        const int p = slot[m], kd = kind[m];
+        uint4 lo, hi;
+        if (kd == kFixed8) {
+            const uint4* src = reinterpret_cast<const uint4*>(blob + L.off_q8 + (size_t)(p - n4) * L.Kp + c * 32);
+            lo = src[0]; hi = src[1];
+        } else {
+            const uint4 raw = *reinterpret_cast<const uint4*>(blob + L.off_q4 + (size_t)p * (L.Kp / 2) + c * 16);
+            uint32_t w[8];
+            if (kd == kPoT4) {
+                expand_pot_chunk(raw, w);
+            } else {
+                // sign-extend the nibbles: (n ^ 8) - 8 per byte, done on 16 * value then shifted with sign
+                expand_fixed4_chunk_x16(raw, w);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const uint32_t x = w[q];
+                    // arithmetic shift right by 4 of each byte: logical shift, then restore the sign bits
+                    const uint32_t s = (x >> 4) & 0x0F0F0F0Fu;
+                    const uint32_t neg = (x >> 7) & 0x01010101u;      // 1 where the byte is negative
+                    w[q] = s | (neg * 0xF0u);
+                }
+            }
+            lo = make_uint4(w[0], w[1], w[2], w[3]); hi = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(wexp + (size_t)m * L.Kp + c * 32);
+        dst[0] = lo; dst[1] = hi;
+    }
+}
+
+cudaError_t launch_expand(const rmsmp_layer& L, const uint8_t* blob, int8_t* wexp, cudaStream_t st)
+{
+    const int64_t total = (int64_t)L.M * (L.Kp >> 5);
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    expand_kernel<<<(unsigned)blocks, 256, 0, st>>>(blob, L, wexp);
     return cudaGetLastError();
 }
 

@@ -62,12 +62,14 @@ struct TensorCfg {
     int nA, nB, nR;        // ring depths: expanded weights, activations, raw weights
     uint32_t raw_bytes;    // one raw stage
     int out_bufs;          // staging buffers per epilogue warp (1 or 2)
+    int pre;               // 1: the A operand comes expanded (int8) from a workspace, no expander work
     uint32_t smem_bytes;
 };
 
 struct Maps {
     CUtensorMap act;                                   // [B][H][W][Cin] activation codes
     CUtensorMap q4, q8;                                // packed weight regions
+    CUtensorMap wexp;                                  // [M][Kp] int8 weights expanded beforehand (pre mode)
     CUtensorMap out_full, out_tail, acc_full, acc_tail;   // bulk stores: 32-row and tail chunks
 };
 
@@ -285,7 +287,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxRing; ++s) {
-            mbar_init(bar_fullA + 8 * s, 4);     // the four warps of one expander group
+            mbar_init(bar_fullA + 8 * s, cfg.pre ? 1 : 4);   // producer (+ bytes), or the four warps of one expander group
             mbar_init(bar_emptyA + 8 * s, 1);    // tcgen05.commit
             mbar_init(bar_fullB + 8 * s, 1);     // producer (+ transaction bytes)
             mbar_init(bar_emptyB + 8 * s, 1);    // tcgen05.commit
@@ -342,13 +344,23 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 int tap = 0, cc = 0;
                 for (int kb = 0; kb < cfg.nkb; ++kb) {
                     const int c0 = cc * 128, koff = tap * p.Cp + c0;
-                    // packed weights of this tile's rows, group by group
-                    if (!mbar_wait_warp(bar_emptyR + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
-                    const uint32_t rbar = bar_fullR + 8 * sr;
-                    if (lane == 0) mbar_arrive_expect_tx(rbar, raw_tx);
-                    __syncwarp();
-                    if (my_map) tma_load_2d(sRaw + sr * cfg.raw_bytes + my_dst, my_map, rbar, my_x8 ? koff : (koff >> 1), my_row);
-                    if (++sr == (uint32_t)cfg.nR) { sr = 0; phR ^= 1; }
+                    if (cfg.pre) {
+                        // weights already expanded: one swizzled 128-row box straight into the A stage
+                        if (!mbar_wait_warp(bar_emptyA + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
+                        if (lane == 0) {
+                            mbar_arrive_expect_tx(bar_fullA + 8 * sr, kABytes);
+                            tma_load_2d(sA + sr * kABytes, &maps.wexp, bar_fullA + 8 * sr, koff, blk * kBlockRows);
+                        }
+                        if (++sr == (uint32_t)cfg.nA) { sr = 0; phR ^= 1; }
+                    } else {
+                        // packed weights of this tile's rows, group by group
+                        if (!mbar_wait_warp(bar_emptyR + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
+                        const uint32_t rbar = bar_fullR + 8 * sr;
+                        if (lane == 0) mbar_arrive_expect_tx(rbar, raw_tx);
+                        __syncwarp();
+                        if (my_map) tma_load_2d(sRaw + sr * cfg.raw_bytes + my_dst, my_map, rbar, my_x8 ? koff : (koff >> 1), my_row);
+                        if (++sr == (uint32_t)cfg.nR) { sr = 0; phR ^= 1; }
+                    }
                     // activation codes
                     if (!mbar_wait_warp(bar_emptyB + 8 * sb, phB ^ 1, abort_flag)) { ok = false; break; }
                     if (lane == 0) {
@@ -403,7 +415,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         const int slot0 = et >> 2;                       // rows slot0 + 32*i of the tile's sorted order
         // tile look-ahead: one tile, or kGroups tiles when every tile is a single k-block
         const int64_t look = (cfg.nkb == 1) ? kGroups : 1;
-        const int64_t total = my_tiles * cfg.nkb;
+        const int64_t total = cfg.pre ? 0 : my_tiles * cfg.nkb;   // nothing to expand in pre mode
         int64_t g = grp;                                 // this CTA's k-block counter
         int64_t tl = g / cfg.nkb;                        // local tile index of g
         int kb = (int)(g - tl * cfg.nkb);
@@ -414,8 +426,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         auto tile_of = [&](int64_t local) -> int64_t { return local < my_tiles ? first + local * step : -1; };
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            cur[i] = make_meta(p, tile_of(tl), slot0 + 32 * i, q);
-            nxt[i] = make_meta(p, tile_of(tl + look), slot0 + 32 * i, q);
+            cur[i] = cfg.pre ? 0u : make_meta(p, tile_of(tl), slot0 + 32 * i, q);
+            nxt[i] = cfg.pre ? 0u : make_meta(p, tile_of(tl + look), slot0 + 32 * i, q);
         }
         while (g < total) {
             const int ksteps = (cc == cfg.cpt - 1) ? cfg.last_ksteps : 4;
@@ -474,7 +486,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
             int shift = 0;
             if (row_ok) {
                 scale = __fmul_rn(__ldg(p.wstep + m), p.act_step);
-                shift = (__ldg(p.kind + m) == kFixed4) ? 4 : 0;
+                shift = (!cfg.pre && __ldg(p.kind + m) == kFixed4) ? 4 : 0;   // expanders store Fixed-4 codes as 16 * value
             }
             if (!mbar_wait_warp(bar_tfull + 8 * ab, (it >> 1) & 1, abort_flag)) break;
             tc_fence_after();
@@ -622,7 +634,8 @@ bool plan(const Problem& p, TensorCfg& c)
 {
     if (p.pix_pitch % 16 != 0 || p.Cin % 16 != 0) return false;
     if ((reinterpret_cast<uintptr_t>(p.act) & 15) != 0) return false;
-    if (p.raw_stage_bytes <= 0) return false;
+    if (!p.wexp && p.raw_stage_bytes <= 0) return false;
+    if (p.wexp && (reinterpret_cast<uintptr_t>(p.wexp) & 15) != 0) return false;
     const int64_t hw = (int64_t)p.Ho * p.Wo;
     if (p.Wo > kTileN || (int64_t)p.Wo * p.stride > 256) return false;
     if (hw <= kTileN) {
@@ -651,6 +664,12 @@ bool plan(const Problem& p, TensorCfg& c)
     c.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.n_mma >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
     c.tail_rows = c.npix & 31;
     c.tma_store = 0;
+    c.pre = p.wexp ? 1 : 0;
+    if (c.pre) {
+        c.nA = 4; c.nB = 4; c.nR = 0; c.raw_bytes = 0; c.out_bufs = 2;
+        c.smem_bytes = (uint32_t)(4 * (kABytes + kBBytes) + kNumEpiWarps * 2 * kWarpStage + 1024 + 64 * kMaxRing);
+        return true;
+    }
     // shared-memory budget: rings as deep as fit
     c.raw_bytes = ((uint32_t)p.raw_stage_bytes + 1023u) & ~1023u;
     const int fixed = 1024 /*alignment*/ + 64 * kMaxRing /*barriers*/;
@@ -707,6 +726,16 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
     };
     if (!make_w(&mp.q4, p.q4, p.nP + p.nF4, p.Kp / 2, 64) || !make_w(&mp.q8, p.q8, p.n8, p.Kp, 128))
         return RMSMP_ERR_CUDA;
+    if (p.wexp) {
+        const cuuint64_t gd[2] = {(cuuint64_t)p.Kp, (cuuint64_t)p.M};
+        const cuuint64_t gs[1] = {(cuuint64_t)p.Kp};
+        const cuuint32_t bx[2] = {128u, (cuuint32_t)kBlockRows};
+        const cuuint32_t es[2] = {1, 1};
+        if (enc(&mp.wexp, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(p.wexp), gd, gs, bx, es,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return RMSMP_ERR_CUDA;
+    }
 
     const bool ld_ok = (p.ld_out % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
                        (!p.acc || (reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);

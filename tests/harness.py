@@ -41,6 +41,16 @@ def unpack(layer, d_packed):
     return vals.cpu().numpy(), perm.cpu().numpy(), ws.cpu().numpy()
 
 
+WORKSPACE = "workspace"     # pseudo-variant: expand once into scratch memory, then the tensor kernel
+
+
+def _workspace(layer, d_packed):
+    torch = torch_mod()
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    return ws
+
+
 def gemm(layer, d_packed, act: np.ndarray, act_step, variant=R.VARIANT_AUTO, out_layout=R.OUT_NM,
          ld_act=None, want_acc=True, canary=True):
     """act: [N][K] int8 host.  Returns (y, acc) as numpy in [N][M] orientation."""
@@ -56,8 +66,12 @@ def gemm(layer, d_packed, act: np.ndarray, act_step, variant=R.VARIANT_AUTO, out
     abuf = torch.full((shape[0] * shape[1] + 2 * pad,), -77777, dtype=torch.int32, device="cuda")
     y = ybuf[pad:pad + shape[0] * shape[1]].view(shape)
     acc = abuf[pad:pad + shape[0] * shape[1]].view(shape)
-    R.rmsmp_gemm_variant(layer, d_packed, a, N, ld, float(np.float32(act_step)), y, shape[1], out_layout,
-                         acc if want_acc else None, variant)
+    if variant == WORKSPACE:
+        R.rmsmp_gemm_workspace(layer, d_packed, _workspace(layer, d_packed), a, N, ld,
+                               float(np.float32(act_step)), y, shape[1], out_layout, acc if want_acc else None)
+    else:
+        R.rmsmp_gemm_variant(layer, d_packed, a, N, ld, float(np.float32(act_step)), y, shape[1], out_layout,
+                             acc if want_acc else None, variant)
     torch.cuda.synchronize()
     assert R.rmsmp_last_device_status(d_packed) == R.OK
     if canary:   # nothing written outside the output
@@ -85,8 +99,12 @@ def conv(layer, d_packed, act: np.ndarray, stride, pad, act_step, variant=R.VARI
     abuf = torch.full((N * M + 2 * cpad,), -77777, dtype=torch.int32, device="cuda")
     y = ybuf[cpad:cpad + N * M].view(shape)
     acc = abuf[cpad:cpad + N * M].view(shape)
-    R.rmsmp_conv_implicit_variant(layer, d_packed, a, B, H, W, stride, pad, float(np.float32(act_step)),
-                                  y, out_layout, acc if want_acc else None, variant)
+    if variant == WORKSPACE:
+        R.rmsmp_conv_implicit_workspace(layer, d_packed, _workspace(layer, d_packed), a, B, H, W, stride, pad,
+                                        float(np.float32(act_step)), y, out_layout, acc if want_acc else None)
+    else:
+        R.rmsmp_conv_implicit_variant(layer, d_packed, a, B, H, W, stride, pad, float(np.float32(act_step)),
+                                      y, out_layout, acc if want_acc else None, variant)
     torch.cuda.synchronize()
     assert R.rmsmp_last_device_status(d_packed) == R.OK
     assert torch.isnan(ybuf[:cpad]).all() and torch.isnan(ybuf[-cpad:]).all()

@@ -14,9 +14,9 @@ from tests import harness as Hn
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [R.VARIANT_SIMPLE, R.VARIANT_SIMT, R.VARIANT_SHIFTADD, R.VARIANT_TENSOR]
+VARIANTS = [R.VARIANT_SIMPLE, R.VARIANT_SIMT, R.VARIANT_SHIFTADD, R.VARIANT_TENSOR, Hn.WORKSPACE]
 VNAME = {R.VARIANT_SIMPLE: "simple", R.VARIANT_SIMT: "simt", R.VARIANT_SHIFTADD: "shiftadd",
-         R.VARIANT_TENSOR: "tensor", R.VARIANT_AUTO: "auto"}
+         R.VARIANT_TENSOR: "tensor", R.VARIANT_AUTO: "auto", Hn.WORKSPACE: "workspace"}
 
 
 def _mixed_map(M, seed, ratio=(60, 35, 5)):
@@ -138,7 +138,7 @@ def test_linear_layer(M, K, N, ratio, variant):
     try:
         y, acc = Hn.gemm(layer, d_packed, act, act_step, variant)
     except R.RmsmpError as e:
-        if e.status == R.ERR_VARIANT and variant == R.VARIANT_TENSOR and K % 16 != 0:
+        if e.status == R.ERR_VARIANT and variant in (R.VARIANT_TENSOR, Hn.WORKSPACE) and K % 16 != 0:
             pytest.skip("tensor variant needs K % 16 == 0")
         raise
     v_ref, ws = O.quantize_rows(W, scheme, bits, alpha)
@@ -146,10 +146,10 @@ def test_linear_layer(M, K, N, ratio, variant):
     _check_layer_outputs(y, acc, acc_ref, ws, act_step, alpha, scheme, bits)
 
 
-@pytest.mark.parametrize("variant", [R.VARIANT_SIMT, R.VARIANT_TENSOR, R.VARIANT_AUTO], ids=lambda v: VNAME[v])
+@pytest.mark.parametrize("variant", [R.VARIANT_SIMT, R.VARIANT_TENSOR, R.VARIANT_AUTO, Hn.WORKSPACE], ids=lambda v: VNAME[v])
 def test_linear_layer_mn_layout_and_padded_ld(variant):
     M, K, N = 140, 160, 70
-    g = synth.rng(74, variant)
+    g = synth.rng(74, variant if isinstance(variant, int) else 9)
     W = synth.weights_normal(g, (M, K))
     scheme, bits = O.assign_rows(W, (60, 35, 5))
     alpha = synth.alpha_rows(W)
@@ -209,7 +209,7 @@ def test_conv_layer(M, Cin, k, stride, pad, B, H, W, variant):
     try:
         y, acc = Hn.conv(layer, d_packed, codes, stride, pad, act_step, variant)
     except R.RmsmpError as e:
-        if e.status == R.ERR_VARIANT and variant == R.VARIANT_TENSOR and Cin % 16 != 0:
+        if e.status == R.ERR_VARIANT and variant in (R.VARIANT_TENSOR, Hn.WORKSPACE) and Cin % 16 != 0:
             pytest.skip("tensor variant needs Cin % 16 == 0")
         raise
     v_ref, ws, acc_ref, y_ref = O.layer_conv(Wt, scheme, bits, alpha, codes, act_step, stride, pad)
