@@ -228,6 +228,27 @@ rmsmp_status rmsmp_conv_implicit_workspace(const rmsmp_layer* layer, const void*
                                            int32_t* d_acc, void* stream);
 
 /*
+ * Linear layer for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a deployment convenience of the library).  Same computation and same results as
+ * rmsmp_expand_weights followed by rmsmp_gemm_workspace, but the scratch for the expanded
+ * weights is a fixed 4 MiB array that is part of the loaded library (each GPU that loads the
+ * library holds it until the process exits), so the call never allocates or frees anything.
+ * Meant for code that runs under a runtime with a fixed memory arena, in a latency-critical
+ * loop, or anywhere else cudaMalloc is off limits.
+ *   - Limit: layer->M * layer->Kp <= 4 MiB (4,194,304 bytes), else RMSMP_ERR_BUFFER_TOO_SMALL.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress); make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps what the last call wrote.  Each call rewrites
+ *     every byte it later reads, so stale contents are harmless, but two calls whose GPU work
+ *     overlaps (different streams, or different host threads) race on it: serialise them.
+ * Arguments and other errors: as rmsmp_gemm.
+ */
+rmsmp_status rmsmp_gemm_builtin_scratch(const rmsmp_layer* layer, const void* d_packed,
+                                        const int8_t* d_act, int64_t N, int64_t ld_act,
+                                        float act_step, float* d_out, int64_t ld_out,
+                                        rmsmp_out_layout out_layout, int32_t* d_acc, void* stream);
+
+/*
  * Read the device status word of a packed buffer (synchronises the stream).  Kernels never
  * trap: a bounded wait that runs out stores RMSMP_ERR_TIMEOUT there and the kernel returns.
  */

@@ -30,7 +30,7 @@ EXPORTS = (
     "rmsmp_unpack_codes", "rmsmp_quantize_act", "rmsmp_gemm", "rmsmp_gemm_variant",
     "rmsmp_conv_implicit", "rmsmp_conv_implicit_variant", "rmsmp_last_device_status",
     "rmsmp_measure_mma_peak", "rmsmp_workspace_bytes", "rmsmp_expand_weights", "rmsmp_gemm_workspace",
-    "rmsmp_conv_implicit_workspace",
+    "rmsmp_conv_implicit_workspace", "rmsmp_gemm_builtin_scratch",
 )
 
 
@@ -94,6 +94,7 @@ def lib() -> C.CDLL:
         L.rmsmp_workspace_bytes.argtypes = [C.POINTER(rmsmp_layer), C.POINTER(C.c_size_t)]
         L.rmsmp_expand_weights.argtypes = [C.POINTER(rmsmp_layer), vp, vp, C.c_size_t, vp]
         L.rmsmp_gemm_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
+        L.rmsmp_gemm_builtin_scratch.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
         L.rmsmp_conv_implicit_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
                                                     f32, vp, i32, vp, vp]
         L.rmsmp_measure_mma_peak.argtypes = [i32, i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
@@ -238,6 +239,15 @@ def rmsmp_conv_implicit_workspace(layer, d_packed, d_workspace, d_act, B: int, H
     _check(lib().rmsmp_conv_implicit_workspace(C.byref(layer), _dp(d_packed), _dp(d_workspace), _dp(d_act),
                                                B, H, W, stride, pad, act_step, _dp(d_out), out_layout,
                                                _dp(d_acc), _stream(stream)), "rmsmp_conv_implicit_workspace")
+
+
+def rmsmp_gemm_builtin_scratch(layer, d_packed, d_act, N: int, ld_act: int, act_step: float, d_out,
+                               ld_out: int, out_layout: int = OUT_NM, d_acc=None, stream=None):
+    """Linear layer through the library's own 4 MiB scratch array: allocates nothing.  For callers
+    that may not call cudaMalloc; calls must not overlap on the GPU (they share the array)."""
+    _check(lib().rmsmp_gemm_builtin_scratch(C.byref(layer), _dp(d_packed), _dp(d_act), N, ld_act,
+                                            act_step, _dp(d_out), ld_out, out_layout, _dp(d_acc),
+                                            _stream(stream)), "rmsmp_gemm_builtin_scratch")
 
 
 def rmsmp_last_device_status(d_packed, stream=None) -> int:
