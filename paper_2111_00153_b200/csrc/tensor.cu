@@ -16,7 +16,8 @@
 //               group by group (PoT, Fixed-4, Fixed-8) but are written to the row of their ORIGINAL
 //               index, so accumulator lanes are in original row order and the output needs no
 //               scatter through the permutation.
-//   warps 10-13 epilogue, one per tensor-memory quarter: tcgen05.ld (next chunk in flight while
+//   warps 10-13 epilogue, one per tensor-memory quarter (in workspace mode the expander warps
+//               have nothing to expand and join the epilogue, three warps per quarter): tcgen05.ld (next chunk in flight while
 //               the current one is processed), undo the x16 of Fixed-4 rows, convert, scale by
 //               wstep*act_step, stage 32 pixels x 32 rows in a private double buffer and write it
 //               with a bulk tensor store.
@@ -63,13 +64,21 @@ struct TensorCfg {
     uint32_t raw_bytes;    // one raw stage
     int out_bufs;          // staging buffers per epilogue warp (1 or 2)
     int pre;               // 1: the A operand comes expanded (int8) from a workspace, no expander work
+    int dup;               // 1 (pre mode, M <= 64): rows 0..63 are loaded twice, into lanes 0..63 and 64..127, so that all
+                           //    four tensor-memory quarters hold valid rows and every epilogue warp has work
+    int epi_warps;         // epilogue warps: 4, or 12 in pre mode (the idle expander warps join)
+    int bk;                // codes per k-block and bytes per operand row in shared memory: 128, or 64 (pre mode,
+                           //    channel counts that would leave half of a 128-byte row empty)
+    int a_bytes, b_bytes;  // one A / B stage
+    int ares;              // 1 (pre mode, one row block, small K): the expanded weights of all k-blocks are loaded once
+                           //    per CTA and stay in shared memory; only activation boxes flow through a ring
     uint32_t smem_bytes;
 };
 
 struct Maps {
     CUtensorMap act;                                   // [B][H][W][Cin] activation codes
     CUtensorMap q4, q8;                                // packed weight regions
-    CUtensorMap wexp;                                  // [M][Kp] int8 weights expanded beforehand (pre mode)
+    CUtensorMap wexp;                                  // [M][Kp] int8 weights expanded beforehand (pre mode); 64-row box when dup
     CUtensorMap out_full, out_tail, acc_full, acc_tail;   // bulk stores: 32-row and tail chunks
 };
 
@@ -151,15 +160,16 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
-// Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+// Shared-memory matrix descriptor: K-major rows of `row_bytes` (128 or 64) with the swizzle of that
+// width; groups of 8 rows are 8*row_bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, int row_bytes)
 {
     uint64_t d = 0;
     d |= (uint64_t)((addr >> 4) & 0x3FFFu);
-    d |= (uint64_t)1 << 16;              // leading byte offset (unused with swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;    // stride byte offset
-    d |= (uint64_t)1 << 46;              // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;              // 128-byte swizzle
+    d |= (uint64_t)1 << 16;                              // leading byte offset (unused with swizzled K-major)
+    d |= (uint64_t)((8 * row_bytes) >> 4) << 32;         // stride byte offset
+    d |= (uint64_t)1 << 46;                              // descriptor version of this architecture
+    d |= (uint64_t)(row_bytes == 128 ? 2 : 4) << 61;     // 128-byte / 64-byte swizzle
     return d;
 }
 __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
@@ -271,10 +281,10 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sA = smem_base;
-    const uint32_t sB = sA + cfg.nA * kABytes;
-    const uint32_t sRaw = sB + cfg.nB * kBBytes;
+    const uint32_t sB = sA + cfg.nA * cfg.a_bytes;
+    const uint32_t sRaw = sB + cfg.nB * cfg.b_bytes;
     const uint32_t sOut = sRaw + cfg.nR * cfg.raw_bytes;
-    const uint32_t sBar = sOut + kNumEpiWarps * cfg.out_bufs * kWarpStage;
+    const uint32_t sBar = sOut + cfg.epi_warps * cfg.out_bufs * kWarpStage;
     // barriers, 8 bytes each
     const uint32_t bar_fullA = sBar, bar_emptyA = sBar + 8 * kMaxRing;
     const uint32_t bar_fullB = sBar + 16 * kMaxRing, bar_emptyB = sBar + 24 * kMaxRing;
@@ -296,7 +306,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_tfull + 8 * b, 1);                  // tcgen05.commit
-            mbar_init(bar_tempty + 8 * b, kNumEpiWarps);      // one arrival per epilogue warp
+            mbar_init(bar_tempty + 8 * b, cfg.epi_warps);     // one arrival per epilogue warp
         }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -321,6 +331,22 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         {
             uint32_t sb = 0, phB = 0, sr = 0, phR = 0;
             bool ok = true;
+            if (cfg.ares && lane == 0 && my_tiles > 0) {
+                // resident weights: every k-block's rows, once
+                mbar_arrive_expect_tx(bar_fullA, (uint32_t)(cfg.nkb * cfg.a_bytes));
+                int tap = 0, cc = 0;
+                for (int kb = 0; kb < cfg.nkb; ++kb) {
+                    const int koff = tap * p.Cp + cc * cfg.bk;
+                    const uint32_t dst = sA + kb * cfg.a_bytes;
+                    if (cfg.dup) {
+                        tma_load_2d(dst, &maps.wexp, bar_fullA, koff, 0);
+                        tma_load_2d(dst + cfg.a_bytes / 2, &maps.wexp, bar_fullA, koff, 0);
+                    } else {
+                        tma_load_2d(dst, &maps.wexp, bar_fullA, koff, 0);
+                    }
+                    if (++cc == cfg.cpt) { cc = 0; ++tap; }
+                }
+            }
             for (int64_t tile = first; tile < cfg.ntiles && ok; tile += step) {
                 const int blk = (int)(tile % p.nblocks);
                 const int64_t nt = tile / p.nblocks;
@@ -343,13 +369,20 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 }
                 int tap = 0, cc = 0;
                 for (int kb = 0; kb < cfg.nkb; ++kb) {
-                    const int c0 = cc * 128, koff = tap * p.Cp + c0;
-                    if (cfg.pre) {
+                    const int c0 = cc * cfg.bk, koff = tap * p.Cp + c0;
+                    if (cfg.ares) {
+                        // weights are resident
+                    } else if (cfg.pre) {
                         // weights already expanded: one swizzled 128-row box straight into the A stage
                         if (!mbar_wait_warp(bar_emptyA + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
                         if (lane == 0) {
-                            mbar_arrive_expect_tx(bar_fullA + 8 * sr, kABytes);
-                            tma_load_2d(sA + sr * kABytes, &maps.wexp, bar_fullA + 8 * sr, koff, blk * kBlockRows);
+                            mbar_arrive_expect_tx(bar_fullA + 8 * sr, cfg.a_bytes);
+                            if (cfg.dup) {
+                                tma_load_2d(sA + sr * cfg.a_bytes, &maps.wexp, bar_fullA + 8 * sr, koff, 0);
+                                tma_load_2d(sA + sr * cfg.a_bytes + cfg.a_bytes / 2, &maps.wexp, bar_fullA + 8 * sr, koff, 0);
+                            } else {
+                                tma_load_2d(sA + sr * cfg.a_bytes, &maps.wexp, bar_fullA + 8 * sr, koff, blk * kBlockRows);
+                            }
                         }
                         if (++sr == (uint32_t)cfg.nA) { sr = 0; phR ^= 1; }
                     } else {
@@ -366,7 +399,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                     if (lane == 0) {
                         const int ti = tap / p.kw, tj = tap - ti * p.kw;
                         mbar_arrive_expect_tx(bar_fullB + 8 * sb, cfg.tx_bytes);
-                        tma_load_4d(sB + sb * kBBytes, &maps.act, bar_fullB + 8 * sb, c0, tj - p.pad,
+                        tma_load_4d(sB + sb * cfg.b_bytes, &maps.act, bar_fullB + 8 * sb, c0, tj - p.pad,
                                     h0 * p.stride + ti - p.pad, b0);
                     }
                     if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; }
@@ -382,7 +415,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         // ---------------------------------------------------------- MMA issuer
         if (lane == 0) {
             uint32_t sa = 0, phA = 0, sb = 0, phB = 0, it = 0;
-            for (int64_t tile = first; tile < cfg.ntiles && !*abort_flag; tile += step, ++it) {
+            bool have_a = !cfg.ares || my_tiles == 0 || mbar_wait(bar_fullA, 0, abort_flag);
+            for (int64_t tile = first; tile < cfg.ntiles && have_a && !*abort_flag; tile += step, ++it) {
                 const uint32_t ab = it & 1;
                 if (!mbar_wait(bar_tempty + 8 * ab, ((it >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after();
@@ -391,13 +425,14 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 int cc = 0;
                 for (int kb = 0; kb < cfg.nkb; ++kb) {
                     if (!mbar_wait(bar_fullB + 8 * sb, phB, abort_flag) ||
-                        !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag)) { ok = false; break; }
+                        (!cfg.ares && !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag))) { ok = false; break; }
                     tc_fence_after();
-                    const int ksteps = (cc == cfg.cpt - 1) ? cfg.last_ksteps : 4;
-                    const uint64_t ad = smem_desc_sw128(sA + sa * kABytes), bd = smem_desc_sw128(sB + sb * kBBytes);
+                    const int ksteps = (cc == cfg.cpt - 1) ? cfg.last_ksteps : (cfg.bk >> 5);
+                    const uint64_t ad = smem_desc_kmajor(sA + (cfg.ares ? (uint32_t)kb : sa) * cfg.a_bytes, cfg.bk),
+                                   bd = smem_desc_kmajor(sB + sb * cfg.b_bytes, cfg.bk);
                     for (int ks = 0; ks < ksteps; ++ks)
                         mma_i8(d_tmem, ad + 2 * ks, bd + 2 * ks, cfg.idesc, (kb | ks) ? 1u : 0u);
-                    mma_commit(bar_emptyA + 8 * sa);
+                    if (!cfg.ares) mma_commit(bar_emptyA + 8 * sa);
                     mma_commit(bar_emptyB + 8 * sb);
                     if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; }
                     if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; }
@@ -407,7 +442,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 mma_commit(bar_tfull + 8 * ab);
             }
         }
-    } else if (warp < 2 + kNumExpWarps) {
+    } else if (!cfg.pre && warp < 2 + kNumExpWarps) {
         // ---------------------------------------------------------- expanders
         const int grp = (warp - 2) >> 2;                 // which k-blocks: g % kGroups == grp
         const int et = ((warp - 2) & 3) * 32 + lane;     // 0..127 inside the group
@@ -434,7 +469,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
             if (!mbar_wait_warp(bar_fullR + 8 * sr, phR, abort_flag)) break;
             if (!mbar_wait_warp(bar_emptyA + 8 * sa, phA ^ 1, abort_flag)) break;
             if (q < ksteps) {
-                const uint32_t rs = sRaw + sr * cfg.raw_bytes, as = sA + sa * kABytes;
+                const uint32_t rs = sRaw + sr * cfg.raw_bytes, as = sA + sa * cfg.a_bytes;
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     if ((cur[i] >> 30) != 3u) expand_task(cur[i], rs, as);
@@ -469,8 +504,16 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         }
     } else {
         // ---------------------------------------------------------- epilogue
-        const int quarter = warp & 3;              // TMEM lanes this warp may read
-        const uint32_t my_stage = sOut + (uint32_t)(warp - (2 + kNumExpWarps)) * (cfg.out_bufs * kWarpStage);
+        // Warp w may read tensor-memory lanes 32*(w%4)..+31.  The warps that share a quarter (one, or
+        // three in pre mode) take alternate 32-pixel chunks; with duplicated rows the two quarters
+        // holding the same rows share the chunks as well.
+        const int quarter = warp & 3;
+        const int ew = cfg.pre ? warp - 2 : warp - (2 + kNumExpWarps);     // 0 .. epi_warps-1
+        const int per_quarter = cfg.epi_warps >> 2;
+        const int row0 = cfg.dup ? (quarter & 1) * 32 : quarter * 32;       // first row (within the block) of this warp
+        const int cstride = cfg.dup ? 2 * per_quarter : per_quarter;
+        const int cfirst = cfg.dup ? (quarter >> 1) * per_quarter + (ew >> 2) : (ew >> 2);
+        const uint32_t my_stage = sOut + (uint32_t)ew * (cfg.out_bufs * kWarpStage);
         uint32_t it = 0, stg_count = 0;
         for (int64_t tile = first; tile < cfg.ntiles; tile += step, ++it) {
             const uint32_t ab = it & 1;
@@ -480,7 +523,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
             if (cfg.tiles_per_image) n0 = ((nt / cfg.tiles_per_image) * p.Ho + (nt % cfg.tiles_per_image) * cfg.th) * (int64_t)p.Wo;
             else n0 = nt * (int64_t)cfg.npix;
             const int nvalid = (int)min((int64_t)cfg.npix, p.N - n0);
-            const int m = blk * kBlockRows + quarter * 32 + lane;
+            const int m = blk * kBlockRows + row0 + lane;
             const bool row_ok = m < p.M;
             float scale = 0.f;
             int shift = 0;
@@ -498,7 +541,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * ab);
             };
-            if (blk * kBlockRows + quarter * 32 >= p.M) {      // no valid row in this quarter
+            if (blk * kBlockRows + row0 >= p.M || cfirst >= nchunks) {      // no valid row, or no chunk, for this warp
                 release_tmem();
                 continue;
             }
@@ -545,7 +588,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                         if (lane == 0) {
                             const CUtensorMap* map = sub ? (tail ? &maps.acc_tail : &maps.acc_full)
                                                          : (tail ? &maps.out_tail : &maps.out_full);
-                            const int cm = blk * kBlockRows + quarter * 32, cn = (int)(n0 + c * 32);
+                            const int cm = blk * kBlockRows + row0, cn = (int)(n0 + c * 32);
                             if (!p.out_mn) tma_store_2d(map, stg, cm, cn); else tma_store_2d(map, stg, cn, cm);
                         }
                     }
@@ -576,19 +619,20 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                     }
                 }
             };
-            // two register sets: the load of chunk c+1 is in flight while chunk c is emitted
+            // two register sets: the load of this warp's next chunk is in flight while the current one is emitted
             uint32_t va[32], vb[32];
-            tmem_ld_issue(taddr, va);
+            tmem_ld_issue(taddr + cfirst * 32, va);
             tmem_ld_wait(va);
-            for (int c = 0; c < nchunks; c += 2) {
-                const bool more1 = c + 1 < nchunks;
-                if (more1) tmem_ld_issue(taddr + (c + 1) * 32, vb); else release_tmem();
+            for (int c = cfirst; c < nchunks; c += 2 * cstride) {
+                const int c1 = c + cstride, c2 = c + 2 * cstride;
+                const bool more1 = c1 < nchunks;
+                if (more1) tmem_ld_issue(taddr + c1 * 32, vb); else release_tmem();
                 emit(va, c);
                 if (more1) {
                     tmem_ld_wait(vb);
-                    const bool more2 = c + 2 < nchunks;
-                    if (more2) tmem_ld_issue(taddr + (c + 2) * 32, va); else release_tmem();
-                    emit(vb, c + 1);
+                    const bool more2 = c2 < nchunks;
+                    if (more2) tmem_ld_issue(taddr + c2 * 32, va); else release_tmem();
+                    emit(vb, c1);
                     if (more2) tmem_ld_wait(va);
                 }
             }
@@ -655,19 +699,36 @@ bool plan(const Problem& p, TensorCfg& c)
     c.npix = c.tb * c.th * p.Wo;
     c.n_mma = (c.npix + 15) / 16 * 16;
     c.ntiles = c.ntiles_n * p.nblocks;
-    c.cpt = (p.Cin + 127) / 128;
+    c.pre = p.wexp ? 1 : 0;
+    // 64-byte k-blocks when a 128-byte row would be at most half used by the (last) channel chunk
+    c.bk = (c.pre && (p.Cin % 128 != 0) && (p.Cin % 128 <= 64)) ? 64 : 128;
+    c.a_bytes = kBlockRows * c.bk;
+    c.b_bytes = kTileN * c.bk;
+    c.cpt = (p.Cin + c.bk - 1) / c.bk;
     c.nkb = p.kh * p.kw * c.cpt;
-    c.last_ksteps = (p.Cin - (c.cpt - 1) * 128 + 31) / 32;
-    c.tx_bytes = (uint32_t)c.npix * 128u;
+    c.last_ksteps = (p.Cin - (c.cpt - 1) * c.bk + 31) / 32;
+    c.tx_bytes = (uint32_t)c.npix * (uint32_t)c.bk;
     // kind::i8: int32 accumulate (bits 4-5 = 2), signed 8-bit A and B (bits 7-9, 10-12 = 1),
     // both K-major, N/8 at bit 17, M/16 at bit 24
     c.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.n_mma >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
     c.tail_rows = c.npix & 31;
     c.tma_store = 0;
-    c.pre = p.wexp ? 1 : 0;
+    c.dup = 0;
+    c.ares = 0;
+    c.epi_warps = kNumEpiWarps;
     if (c.pre) {
-        c.nA = 4; c.nB = 4; c.nR = 0; c.raw_bytes = 0; c.out_bufs = 2;
-        c.smem_bytes = (uint32_t)(4 * (kABytes + kBBytes) + kNumEpiWarps * 2 * kWarpStage + 1024 + 64 * kMaxRing);
+        c.nA = (c.bk == 64) ? 6 : 3; c.nB = (c.bk == 64) ? 8 : 4; c.nR = 0; c.raw_bytes = 0; c.out_bufs = 1;
+        c.epi_warps = kNumExpWarps + kNumEpiWarps;
+        c.dup = (p.M <= 64) ? 1 : 0;
+        if (p.nblocks == 1 && (int64_t)c.nkb * c.a_bytes <= 72 * 1024) {
+            c.ares = 1;
+            c.nA = c.nkb;
+            const int64_t left = kSmemLimit - (1024 + 64 * kMaxRing) - (int64_t)c.nkb * c.a_bytes -
+                                 (int64_t)c.epi_warps * kWarpStage;
+            c.nB = (int)std::min<int64_t>(kMaxRing, left / c.b_bytes);
+        }
+        c.smem_bytes = (uint32_t)(c.nA * c.a_bytes + c.nB * c.b_bytes + c.epi_warps * c.out_bufs * kWarpStage + 1024 +
+                                  64 * kMaxRing);
         return true;
     }
     // shared-memory budget: rings as deep as fit
@@ -706,11 +767,11 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
         const cuuint64_t gdim[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
         const cuuint64_t gstr[3] = {(cuuint64_t)p.pix_pitch, (cuuint64_t)p.pix_pitch * p.W,
                                     (cuuint64_t)p.pix_pitch * p.W * p.H};
-        const cuuint32_t box[4] = {128u, (cuuint32_t)(p.Wo * p.stride), (cuuint32_t)(c.th * p.stride), (cuuint32_t)c.tb};
+        const cuuint32_t box[4] = {(cuuint32_t)c.bk, (cuuint32_t)(p.Wo * p.stride), (cuuint32_t)(c.th * p.stride), (cuuint32_t)c.tb};
         const cuuint32_t estr[4] = {1u, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1u};
         if (enc(&mp.act, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(p.act), gdim, gstr, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                CU_TENSOR_MAP_INTERLEAVE_NONE, c.bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return RMSMP_ERR_CUDA;
     }
     // packed weight regions: rows of Kp/2 (4-bit) and Kp (8-bit) bytes, boxes of 16 rows x one k-block
@@ -729,10 +790,11 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
     if (p.wexp) {
         const cuuint64_t gd[2] = {(cuuint64_t)p.Kp, (cuuint64_t)p.M};
         const cuuint64_t gs[1] = {(cuuint64_t)p.Kp};
-        const cuuint32_t bx[2] = {128u, (cuuint32_t)kBlockRows};
+        const cuuint32_t bx[2] = {(cuuint32_t)c.bk, (cuuint32_t)(c.dup ? kBlockRows / 2 : kBlockRows)};
         const cuuint32_t es[2] = {1, 1};
         if (enc(&mp.wexp, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(p.wexp), gd, gs, bx, es,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, c.bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return RMSMP_ERR_CUDA;
     }
