@@ -261,14 +261,32 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restri
     const size_t tid = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
     const size_t nthr = (size_t)gridDim.x * blockDim.x;
     if (vec) {
-        // 16 values per thread step: four 128-bit loads, one 128-bit store
+        // 32 values per thread step: eight 128-bit loads in flight, then two 128-bit stores
         const size_t n16 = count / 16;
-        for (size_t i = tid; i < n16; i += nthr) {
+        const size_t n32 = count / 32;
+        for (size_t i = tid; i < n32; i += nthr) {
+            const float4* src = reinterpret_cast<const float4*>(x) + i * 8;
+            float4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = __ldcs(src + j);
+            uint32_t w[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                w[j] = (uint32_t)(act_code(v[j].x, alpha, kind) & 0xFF) |
+                       ((uint32_t)(act_code(v[j].y, alpha, kind) & 0xFF) << 8) |
+                       ((uint32_t)(act_code(v[j].z, alpha, kind) & 0xFF) << 16) |
+                       ((uint32_t)(act_code(v[j].w, alpha, kind) & 0xFF) << 24);
+            uint4* dst = reinterpret_cast<uint4*>(codes) + i * 2;
+            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+        if ((n16 & 1) && tid == 0) {              // one 16-value group left over
+            const size_t i = n16 - 1;
             const float4* src = reinterpret_cast<const float4*>(x) + i * 4;
             uint32_t w[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                float4 v = __ldcs(src + j);
+                float4 v = src[j];
                 w[j] = (uint32_t)(act_code(v.x, alpha, kind) & 0xFF) |
                        ((uint32_t)(act_code(v.y, alpha, kind) & 0xFF) << 8) |
                        ((uint32_t)(act_code(v.z, alpha, kind) & 0xFF) << 16) |
@@ -286,7 +304,7 @@ cudaError_t launch_quantize_act(const float* x, size_t count, float alpha, int k
                                 cudaStream_t st)
 {
     int vec = ((reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(codes) & 15) == 0);
-    size_t steps = vec ? (count + 15) / 16 : count;
+    size_t steps = vec ? (count + 31) / 32 : count;
     size_t blocks = (steps + 255) / 256;
     const size_t cap = 148 * 32;
     if (blocks > cap) blocks = cap;

@@ -1,0 +1,171 @@
+"""GPU parity at the sizes of the five workload configurations, in the launch configuration the
+benchmark uses (workspace variant, [N][M] output), against the CPU oracle.
+
+Small enough cases are compared in full; the large ones on randomly sampled outputs the oracle
+computes one by one (the integer sums are exact, so a sample that covers every row kind, image
+borders and tile tails is as strict per element as the full comparison).
+"""
+import numpy as np
+import pytest
+
+from oracle import rmsmp_oracle as O
+from paper_2111_00153_b200 import binding as R
+from paper_2111_00153_b200 import synth
+from tests import harness as Hn
+
+pytestmark = pytest.mark.gpu
+
+
+def _expected(acc, ws, act_step):
+    return O.epilogue(acc, ws, act_step)
+
+
+def _run_conv_device(W, scheme, bits, alpha, x, stride, pad, kind, workspace=True):
+    """fp32 weights / activations on the host -> (codes, step, y) through the C ABI."""
+    import torch
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    dx = torch.from_numpy(x).cuda()
+    codes = torch.empty(x.shape, dtype=torch.int8, device="cuda")
+    step = R.rmsmp_quantize_act(dx, dx.numel(), synth.ALPHA_ACT, kind, codes)
+    B, H, Wd, _ = x.shape
+    Ho, Wo = O.conv_out_hw(H, Wd, layer.kh, layer.kw, stride, pad)
+    y = torch.full((B * Ho * Wo, layer.M), float("nan"), dtype=torch.float32, device="cuda")
+    if workspace:
+        ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+        R.rmsmp_expand_weights(layer, d_packed, ws)
+        R.rmsmp_conv_implicit_workspace(layer, d_packed, ws, codes, B, H, Wd, stride, pad, step, y)
+    else:
+        R.rmsmp_conv_implicit_variant(layer, d_packed, codes, B, H, Wd, stride, pad, step, y, R.OUT_NM, None,
+                                      R.VARIANT_TENSOR)
+    torch.cuda.synchronize()
+    assert R.rmsmp_last_device_status(d_packed) == R.OK
+    return codes.cpu().numpy(), np.float32(step), y.cpu().numpy()
+
+
+# ------------------------------------------------------------------ config 2: one ResNet conv, full
+
+@pytest.mark.parametrize("workspace", [True, False], ids=["workspace", "smem"])
+def test_config2_conv256_14x14_batch32_full(workspace):
+    L = synth.CONFIG2_CONV
+    g = synth.rng(2, 0)
+    W = synth.weights_kaiming(g, L.M, L.Cin, L.k, L.k)
+    x = synth.act_halfnormal(g, (32, L.H, L.H, L.Cin))
+    scheme, bits = O.assign_rows(W, synth.RATIO_RMSMP1)
+    assert (int((scheme == 0).sum()), int(((scheme == 1) & (bits == 4)).sum()), int((bits == 8).sum())) == (154, 89, 13)
+    alpha = synth.alpha_rows(W)
+    codes, step, y = _run_conv_device(W, scheme, bits, alpha, x, L.stride, L.pad, R.ACT_U4, workspace)
+    c_ref, s_ref = O.quantize_act(x, synth.ALPHA_ACT, O.ACT_U4)
+    assert np.array_equal(codes, c_ref) and step == s_ref
+    _, ws, acc, y_ref = O.layer_conv(W, scheme, bits, alpha, c_ref, s_ref, L.stride, L.pad)
+    assert np.array_equal(y.view(np.uint32), y_ref.reshape(-1, L.M).view(np.uint32))
+
+
+# ------------------------------------------------------------------ config 3: BERT-base linears, N = 4096
+
+@pytest.mark.parametrize("name,M,K", synth.BERT_BASE_LINEARS)
+def test_config3_bert_base_linear(name, M, K):
+    import torch
+    N = synth.BERT_BASE_TOKENS
+    g = synth.rng(3, M + K)
+    W = synth.weights_normal(g, (M, K))
+    x = synth.act_normal(g, (N, K))
+    scheme, bits = O.assign_rows(W, synth.RATIO_RMSMP1)
+    alpha = synth.alpha_rows(W)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    dx = torch.from_numpy(x).cuda()
+    codes = torch.empty((N, K), dtype=torch.int8, device="cuda")
+    step = R.rmsmp_quantize_act(dx, dx.numel(), synth.ALPHA_ACT, R.ACT_S4, codes)
+    y = torch.empty((N, M), dtype=torch.float32, device="cuda")
+    acc = torch.empty((N, M), dtype=torch.int32, device="cuda")
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    R.rmsmp_gemm_workspace(layer, d_packed, ws, codes, N, K, step, y, M, R.OUT_NM, acc)
+    y2 = torch.empty((N, M), dtype=torch.float32, device="cuda")
+    R.rmsmp_gemm(layer, d_packed, codes, N, K, step, y2, M)           # the in-shared-memory expansion path
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+    c_ref, s_ref = O.quantize_act(x, synth.ALPHA_ACT, O.ACT_S4)
+    assert np.array_equal(codes.cpu().numpy(), c_ref) and np.float32(step) == s_ref
+    v_ref, wstep = O.quantize_rows(W, scheme, bits, alpha)
+    if M * K * N <= 3e9:                                   # attn_out: everything
+        acc_ref = O.matmul(v_ref, c_ref)
+        assert np.array_equal(acc.cpu().numpy(), acc_ref)
+        assert np.array_equal(y.cpu().numpy().view(np.uint32), _expected(acc_ref, wstep, s_ref).view(np.uint32))
+    else:                                                   # sampled outputs, every row at least once
+        r = np.random.default_rng(M)
+        n_idx = np.concatenate([r.integers(0, N, 40000), r.integers(0, N, M), [0, N - 1, N - 1]])
+        m_idx = np.concatenate([r.integers(0, M, 40000), np.arange(M), [0, M - 1, 0]]).astype(np.int32)
+        pts = O.matmul_points(v_ref, c_ref, n_idx, m_idx)
+        assert np.array_equal(acc.cpu().numpy()[n_idx, m_idx], pts)
+        c = (wstep[m_idx] * s_ref).astype(np.float32)
+        want = (pts.astype(np.float32) * c).astype(np.float32)
+        assert np.array_equal(y.cpu().numpy()[n_idx, m_idx].view(np.uint32), want.view(np.uint32))
+
+
+# ------------------------------------------------------------------ config 4: the ResNet-18 stack
+
+@pytest.mark.parametrize("L", synth.resnet18_convs(), ids=lambda L: L.name)
+def test_config4_resnet18_layer_batch4_full(L):
+    g = synth.rng(4, L.M + L.Cin + L.k)
+    W = synth.weights_kaiming(g, L.M, L.Cin, L.k, L.k)
+    x = synth.act_halfnormal(g, (4, L.H, L.H, L.Cin))
+    scheme, bits = R.rmsmp_assign_rows(W, synth.RATIO_RMSMP1)
+    alpha = synth.alpha_rows(W)
+    codes, step, y = _run_conv_device(W, scheme, bits, alpha, x, L.stride, L.pad, R.ACT_U4)
+    _, ws, acc, y_ref = O.layer_conv(W, scheme, bits, alpha, codes, step, L.stride, L.pad)
+    assert np.array_equal(y.view(np.uint32), y_ref.reshape(-1, L.M).view(np.uint32))
+
+
+BIG = [L for L in synth.resnet18_convs() if L.name in
+       ("l1.conv3x3", "l2.conv3x3_s2", "l2.down1x1_s2", "l3.conv3x3", "l4.conv3x3")]
+
+
+@pytest.mark.parametrize("L", BIG, ids=lambda L: L.name)
+def test_config4_resnet18_layer_batch256_sampled(L):
+    B = 256
+    g = synth.rng(4, 7 * L.M + L.H)
+    W = synth.weights_kaiming(g, L.M, L.Cin, L.k, L.k)
+    x = synth.act_halfnormal(g, (B, L.H, L.H, L.Cin))
+    scheme, bits = R.rmsmp_assign_rows(W, synth.RATIO_RMSMP1)
+    alpha = synth.alpha_rows(W)
+    codes, step, y = _run_conv_device(W, scheme, bits, alpha, x, L.stride, L.pad, R.ACT_U4)
+    # activation codes: a sample against the oracle's quantizer
+    r = np.random.default_rng(L.M + L.H)
+    flat = r.integers(0, x.size, 200000)
+    c_ref, s_ref = O.quantize_act(x.ravel()[flat], synth.ALPHA_ACT, O.ACT_U4)
+    assert np.array_equal(codes.ravel()[flat], c_ref) and step == s_ref
+    # outputs: random points, every row, the four image corners of first and last image, last pixels
+    N = B * L.Ho * L.Ho
+    hw = L.Ho * L.Ho
+    corners = [0, L.Ho - 1, hw - L.Ho, hw - 1]
+    special = np.array([c for c in corners] + [(B - 1) * hw + c for c in corners] + [N - 1, N - 2])
+    n_idx = np.concatenate([r.integers(0, N, 60000), r.integers(0, N, L.M), np.repeat(special, 2)])
+    m_idx = np.concatenate([r.integers(0, L.M, 60000), np.arange(L.M),
+                            np.tile([0, L.M - 1], special.size)]).astype(np.int32)
+    v_ref, wstep = O.quantize_rows(W.reshape(L.M, -1), scheme, bits, alpha)
+    pts = O.conv_points(v_ref.reshape(W.shape), codes, L.stride, L.pad, n_idx, m_idx)
+    c = (wstep[m_idx] * step).astype(np.float32)
+    want = (pts.astype(np.float32) * c).astype(np.float32)
+    assert np.array_equal(y[n_idx, m_idx].view(np.uint32), want.view(np.uint32))
+    assert not np.isnan(y).any()                         # every output was written
+
+
+# ------------------------------------------------------------------ config 5: weight-bound small-N sweep
+
+@pytest.mark.parametrize("ratio", synth.RATIO_SWEEP, ids=lambda r: "%d-%d-%d" % r)
+@pytest.mark.parametrize("N", synth.BERT_LARGE_TOKENS)
+@pytest.mark.parametrize("name,M,K", synth.BERT_LARGE_LINEARS)
+def test_config5_bert_large_small_batch(name, M, K, N, ratio):
+    g = synth.rng(5, M // 64 + K // 32 + N + ratio[0])
+    W = synth.weights_normal(g, (M, K))
+    scheme, bits = O.assign_rows(W, ratio)
+    alpha = synth.alpha_rows(W)
+    act = synth.act_codes_uniform(g, (N, K))
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    v_ref, wstep = O.quantize_rows(W, scheme, bits, alpha)
+    acc_ref = O.matmul(v_ref, act)
+    y_ref = _expected(acc_ref, wstep, np.float32(0.05))
+    for variant in (R.VARIANT_AUTO, R.VARIANT_SHIFTADD, R.VARIANT_TENSOR):
+        y, acc = Hn.gemm(layer, d_packed, act, 0.05, variant)
+        assert np.array_equal(acc, acc_ref)
+        assert np.array_equal(y.view(np.uint32), y_ref.view(np.uint32))
