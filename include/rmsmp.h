@@ -11,6 +11,8 @@
  *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller owns every
  *     buffer; the library allocates no device memory and keeps no reference after a call
  *     returns (work already queued on the stream keeps using the buffers until it is done).
+ *     The only memory it obtains by itself is 2 MiB of pinned HOST memory per device, on the first
+ *     rmsmp_quantize_pack, used to upload the layer metadata without stalling the stream.
  *   - `stream` is a cudaStream_t passed as void* (0 = default stream).  All device work is
  *     asynchronous on it.
  *   - Every function returns an rmsmp_status and never throws, aborts or prints.  Everything

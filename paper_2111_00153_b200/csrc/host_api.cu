@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <vector>
 #include "common.cuh"
 
@@ -42,6 +43,57 @@ rmsmp_status check_arch()
         have[dev] = true;
     }
     return cached_major[dev] == 10 ? RMSMP_OK : RMSMP_ERR_ARCH;
+}
+
+// Pinned host staging for the metadata upload of rmsmp_quantize_pack.  A copy from pageable memory
+// makes the host wait for the stream; from pinned memory it is asynchronous.  One small ring of
+// slots per device, created on first use (host memory only; no device memory is ever allocated);
+// an event per slot tells when its last copy has left.  If pinned memory cannot be had, or the
+// metadata is larger than a slot, the pageable path is used.
+constexpr size_t kStageSlotBytes = 64 * 1024;
+constexpr int kStageSlots = 32;
+struct StageRing {
+    bool tried = false;
+    uint8_t* base = nullptr;
+    cudaEvent_t ev[kStageSlots];
+    bool used[kStageSlots];
+    int next = 0;
+};
+StageRing g_stage[64];
+std::mutex g_stage_mutex;
+
+// Copies `bytes` of metadata to the device through a pinned slot; false = caller uses the pageable path.
+bool staged_upload(void* d_dst, const void* h_src, size_t bytes, cudaStream_t st)
+{
+    if (bytes > kStageSlotBytes) return false;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return false; }
+    std::lock_guard<std::mutex> lock(g_stage_mutex);
+    StageRing& r = g_stage[dev];
+    if (!r.tried) {
+        r.tried = true;
+        void* ptr = nullptr;
+        if (cudaHostAlloc(&ptr, kStageSlotBytes * kStageSlots, cudaHostAllocDefault) != cudaSuccess) {
+            cudaGetLastError();
+        } else {
+            bool ok = true;
+            for (int i = 0; i < kStageSlots; ++i) {
+                r.used[i] = false;
+                if (cudaEventCreateWithFlags(&r.ev[i], cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); ok = false; break; }
+            }
+            if (ok) r.base = static_cast<uint8_t*>(ptr); else cudaFreeHost(ptr);
+        }
+    }
+    if (!r.base) return false;
+    const int slot = r.next;
+    r.next = (r.next + 1) % kStageSlots;
+    if (r.used[slot] && cudaEventSynchronize(r.ev[slot]) != cudaSuccess) { cudaGetLastError(); return false; }
+    uint8_t* h = r.base + (size_t)slot * kStageSlotBytes;
+    std::memcpy(h, h_src, bytes);
+    if (cudaMemcpyAsync(d_dst, h, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (cudaEventRecord(r.ev[slot], st) != cudaSuccess) { cudaGetLastError(); return false; }
+    r.used[slot] = true;
+    return true;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
@@ -236,7 +288,8 @@ rmsmp_status rmsmp_quantize_pack(const float* d_W, rmsmp_w_layout w_layout, cons
         wstep[r] = h_alpha[r] / q;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(d_packed, meta.data(), meta.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    if (!staged_upload(d_packed, meta.data(), meta.size(), st) &&
+        cudaMemcpyAsync(d_packed, meta.data(), meta.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return RMSMP_ERR_CUDA;
     }

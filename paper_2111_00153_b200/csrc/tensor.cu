@@ -324,8 +324,59 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
     const int64_t first = blockIdx.x, step = gridDim.x;
     const int64_t my_tiles = (cfg.ntiles > first) ? (cfg.ntiles - first + step - 1) / step : 0;
 
-    if (warp == 0) {
-        // ---------------------------------------------------------- TMA producer
+    // Workspace mode splits the producer: one thread can start a bulk tensor copy only every few
+    // hundred cycles, so the activation boxes and the weight boxes are issued by two different warps.
+    const bool pre_b_producer = cfg.pre && warp == 0;
+    const bool pre_a_producer = cfg.pre && !cfg.ares && warp == 2;
+    if (pre_b_producer || pre_a_producer) {
+        if (lane == 0) {
+            if (pre_b_producer && cfg.ares && my_tiles > 0) {
+                // resident weights: every k-block's rows, once
+                mbar_arrive_expect_tx(bar_fullA, (uint32_t)(cfg.nkb * cfg.a_bytes));
+                int tap = 0, cc = 0;
+                for (int kb = 0; kb < cfg.nkb; ++kb) {
+                    const int koff = tap * p.Cp + cc * cfg.bk;
+                    const uint32_t dst = sA + kb * cfg.a_bytes;
+                    tma_load_2d(dst, &maps.wexp, bar_fullA, koff, 0);
+                    if (cfg.dup) tma_load_2d(dst + cfg.a_bytes / 2, &maps.wexp, bar_fullA, koff, 0);
+                    if (++cc == cfg.cpt) { cc = 0; ++tap; }
+                }
+            }
+            const uint32_t nring = pre_b_producer ? (uint32_t)cfg.nB : (uint32_t)cfg.nA;
+            const uint32_t bar_e = pre_b_producer ? bar_emptyB : bar_emptyA;
+            const uint32_t bar_f = pre_b_producer ? bar_fullB : bar_fullA;
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (int64_t tile = first; tile < cfg.ntiles && ok; tile += step) {
+                const int64_t nt = tile / p.nblocks;
+                const int blk = (int)(tile - nt * p.nblocks);
+                int b0, h0;
+                if (cfg.tiles_per_image) { b0 = (int)(nt / cfg.tiles_per_image); h0 = (int)(nt % cfg.tiles_per_image) * cfg.th; }
+                else { b0 = (int)(nt * cfg.tb); h0 = 0; }
+                const int row_a = cfg.dup ? 0 : blk * kBlockRows;
+                const int y_base = h0 * p.stride - p.pad;
+                int tap = 0, cc = 0, ti = 0, tj = 0;
+                for (int kb = 0; kb < cfg.nkb; ++kb) {
+                    if (!mbar_wait(bar_e + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
+                    if (pre_b_producer) {
+                        mbar_arrive_expect_tx(bar_f + 8 * s, cfg.tx_bytes);
+                        tma_load_4d(sB + s * cfg.b_bytes, &maps.act, bar_f + 8 * s, cc * cfg.bk, tj - p.pad, y_base + ti, b0);
+                    } else {
+                        const int koff = tap * p.Cp + cc * cfg.bk;
+                        mbar_arrive_expect_tx(bar_f + 8 * s, cfg.a_bytes);
+                        tma_load_2d(sA + s * cfg.a_bytes, &maps.wexp, bar_f + 8 * s, koff, row_a);
+                        if (cfg.dup) tma_load_2d(sA + s * cfg.a_bytes + cfg.a_bytes / 2, &maps.wexp, bar_f + 8 * s, koff, row_a);
+                    }
+                    if (++s == nring) { s = 0; ph ^= 1; }
+                    if (++cc == cfg.cpt) { cc = 0; ++tap; if (++tj == p.kw) { tj = 0; ++ti; } }
+                }
+            }
+            if (!ok) {
+                for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land
+            }
+        }
+    } else if (warp == 0) {
+        // ---------------------------------------------------------- TMA producer (shared-memory expansion mode)
         // The whole warp takes part: lane 0 waits on the barriers and fetches the activation box,
         // the weight boxes of a k-block are issued by one lane each.
         {
@@ -508,11 +559,14 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         // three in pre mode) take alternate 32-pixel chunks; with duplicated rows the two quarters
         // holding the same rows share the chunks as well.
         const int quarter = warp & 3;
-        const int ew = cfg.pre ? warp - 2 : warp - (2 + kNumExpWarps);     // 0 .. epi_warps-1
-        const int per_quarter = cfg.epi_warps >> 2;
+        const int first_epi = kThreads / 32 - cfg.epi_warps;               // epilogue warps are the last epi_warps warps
+        const int ew = warp - first_epi;                                   // 0 .. epi_warps-1
+        // how many epilogue warps share a quarter, and this warp's rank among them
+        auto count_q = [&](int q) { const int f = first_epi + ((q - first_epi) & 3); return (kThreads / 32 - 1 - f) / 4 + 1; };
+        const int my_rank = (warp - (first_epi + ((quarter - first_epi) & 3))) >> 2;
         const int row0 = cfg.dup ? (quarter & 1) * 32 : quarter * 32;       // first row (within the block) of this warp
-        const int cstride = cfg.dup ? 2 * per_quarter : per_quarter;
-        const int cfirst = cfg.dup ? (quarter >> 1) * per_quarter + (ew >> 2) : (ew >> 2);
+        const int cstride = cfg.dup ? count_q(quarter & 1) + count_q((quarter & 1) + 2) : count_q(quarter);
+        const int cfirst = (cfg.dup && (quarter >> 1)) ? count_q(quarter & 1) + my_rank : my_rank;
         const uint32_t my_stage = sOut + (uint32_t)ew * (cfg.out_bufs * kWarpStage);
         uint32_t it = 0, stg_count = 0;
         for (int64_t tile = first; tile < cfg.ntiles; tile += step, ++it) {
@@ -718,10 +772,11 @@ bool plan(const Problem& p, TensorCfg& c)
     c.epi_warps = kNumEpiWarps;
     if (c.pre) {
         c.nA = (c.bk == 64) ? 6 : 3; c.nB = (c.bk == 64) ? 8 : 4; c.nR = 0; c.raw_bytes = 0; c.out_bufs = 1;
-        c.epi_warps = kNumExpWarps + kNumEpiWarps;
+        c.epi_warps = kNumExpWarps + kNumEpiWarps - 1;   // warp 2 fetches the weights (unless they are resident)
         c.dup = (p.M <= 64) ? 1 : 0;
         if (p.nblocks == 1 && (int64_t)c.nkb * c.a_bytes <= 72 * 1024) {
             c.ares = 1;
+            c.epi_warps = kNumExpWarps + kNumEpiWarps;
             c.nA = c.nkb;
             const int64_t left = kSmemLimit - (1024 + 64 * kMaxRing) - (int64_t)c.nkb * c.a_bytes -
                                  (int64_t)c.epi_warps * kWarpStage;
