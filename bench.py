@@ -386,6 +386,105 @@ def run_reference(args):
     }))
 
 
+# ---------------------------------------------------------------------------- variant comparison
+
+def run_suite(args):
+    """Side-by-side timing of the contraction variants on the five workload configurations.
+    Prints one JSON line per (shape, variant) and a markdown table; not the headline number."""
+    import torch
+    from paper_2111_00153_b200 import binding as R
+    torch.cuda.set_device(0)
+    peaks, peak_src = load_peaks()
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    i8_peak, _ = R.rmsmp_measure_mma_peak(status, False, 256, 20000)
+    bf_peak, _ = R.rmsmp_measure_mma_peak(status, True, 256, 20000)
+    print(json.dumps({"suite": "peaks", "int8_mma_tops_measured": i8_peak, "bf16_mma_tops_measured": bf_peak,
+                      "hbm_gbs": peaks["hbm_gbs"], "hbm_source": peak_src}))
+    rows = []
+
+    def timed(fn, iters):
+        for _ in range(3):
+            fn(0)
+        torch.cuda.synchronize()
+        best = []
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(iters):
+                fn(i)
+            b.record()
+            torch.cuda.synchronize()
+            best.append(a.elapsed_time(b) / iters)
+        return float(np.median(best)) * 1e3      # microseconds
+
+    def prep(M, Cin, k, ratio, seed, conv):
+        g = synth.rng(6, seed)
+        W = synth.weights_kaiming(g, M, Cin, k, k) if conv else synth.weights_normal(g, (M, Cin)).reshape(M, Cin, 1, 1)
+        scheme, bits = R.rmsmp_assign_rows(W, ratio)
+        lay = R.rmsmp_layer_init(M, Cin, k, k, scheme, bits)
+        pk = torch.empty(lay.packed_bytes, dtype=torch.uint8, device="cuda")
+        R.rmsmp_quantize_pack(torch.from_numpy(W).cuda(), R.W_CONV_OIHW, lay, scheme, bits, synth.alpha_rows(W),
+                              R.POT_NEAREST, pk)
+        ws = torch.empty(R.rmsmp_workspace_bytes(lay), dtype=torch.int8, device="cuda")
+        R.rmsmp_expand_weights(lay, pk, ws)
+        return lay, pk, ws
+
+    VAR = (("tensor_smem", R.VARIANT_TENSOR), ("tensor_workspace", "ws"), ("simt_dp4a", R.VARIANT_SIMT),
+           ("shift_add", R.VARIANT_SHIFTADD))
+
+    def bench_shape(cfg, name, M, Cin, k, stride, pad, B, H, ratio=RATIO, pool=1, only=None, iters=20):
+        conv = k > 1 or H > 1
+        inst = [prep(M, Cin, k, ratio, 17 * i + M, conv) for i in range(pool)]
+        Ho = (H + 2 * pad - k) // stride + 1
+        N = B * Ho * Ho
+        act = torch.randint(0, 16, (B, H, H, Cin), dtype=torch.int8, device="cuda")
+        y = torch.empty((N, M), dtype=torch.float32, device="cuda")
+        lay0 = inst[0][0]
+        ops = 2 * M * Cin * k * k * N
+        pix_in = Ho * Ho if (k == 1 and stride > 1) else H * H
+        alg = (lay0.nP + lay0.nF4) * lay0.K // 2 + lay0.n8 * lay0.K + 8 * M + B * pix_in * Cin + 4 * N * M
+        for vname, v in VAR:
+            if only and vname not in only:
+                continue
+            def fn(i, v=v):
+                lay, pk, ws = inst[i % pool]
+                if v == "ws":
+                    R.rmsmp_conv_implicit_workspace(lay, pk, ws, act, B, H, H, stride, pad, 0.1, y, R.OUT_NM, None)
+                else:
+                    R.rmsmp_conv_implicit_variant(lay, pk, act, B, H, H, stride, pad, 0.1, y, R.OUT_NM, None, v)
+            try:
+                us = timed(fn, iters if v in ("ws", R.VARIANT_TENSOR) or ops < 2e10 else 3)
+            except R.RmsmpError as e:
+                print(json.dumps({"suite": cfg, "shape": name, "variant": vname, "error": str(e)}))
+                continue
+            rec = {"suite": cfg, "shape": name, "M": M, "K": Cin * k * k, "N": N, "ratio": list(ratio), "variant": vname,
+                   "us": us, "tops": ops / us / 1e6, "gbs": alg / us / 1e3, "frac_int8_peak": ops / us / 1e6 / i8_peak,
+                   "frac_hbm": alg / us / 1e3 / peaks["hbm_gbs"], "weights": "cold pool of %d" % pool if pool > 1 else "warm"}
+            rows.append(rec)
+            print(json.dumps(rec))
+
+    bench_shape("config1", "linear 256x512 N=64", 256, 512, 1, 1, 0, 64, 1)
+    L = synth.CONFIG2_CONV
+    bench_shape("config2", "conv 256->256 3x3 14x14 B=32", L.M, L.Cin, 3, 1, 1, 32, 14)
+    for nm, M, K in synth.BERT_BASE_LINEARS:
+        bench_shape("config3", "bert-base %s %dx%d N=4096" % (nm, M, K), M, K, 1, 1, 0, 4096, 1)
+    for L in synth.resnet18_convs():
+        if L.name in ("l1.conv3x3", "l2.conv3x3", "l2.down1x1_s2", "l3.conv3x3", "l4.conv3x3"):
+            bench_shape("config4", "resnet18 %s B=256" % L.name, L.M, L.Cin, L.k, L.stride, L.pad, 256, L.H)
+    for nm, M, K in synth.BERT_LARGE_LINEARS:
+        for N in synth.BERT_LARGE_TOKENS:
+            bench_shape("config5", "bert-large %s %dx%d N=%d" % (nm, M, K, N), M, K, 1, 1, 0, N, 1, pool=24,
+                        only=("simt_dp4a", "shift_add") if N < 32 else None, iters=48)
+    for ratio in synth.RATIO_SWEEP:
+        bench_shape("config5", "bert-large ffn1 4096x1024 N=8 ratio %d:%d:%d" % ratio, 4096, 1024, 1, 1, 0, 8, 1,
+                    ratio=ratio, pool=24, only=("simt_dp4a", "shift_add"), iters=48)
+    print("\n| config | shape | variant | us | TOPS | GB/s | of INT8 peak | of HBM |")
+    print("|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        print("| %s | %s | %s | %.1f | %.1f | %.0f | %.1f %% | %.1f %% |" % (
+            r["suite"], r["shape"], r["variant"], r["us"], r["tops"], r["gbs"], 100 * r["frac_int8_peak"], 100 * r["frac_hbm"]))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -400,13 +499,17 @@ def main():
     ap.add_argument("--variant", default="workspace", choices=["workspace", "smem"],
                     help="tensor-core path: expand the weight codes once into scratch memory (default) "
                          "or in shared memory per tile")
+    ap.add_argument("--suite", action="store_true",
+                    help="side-by-side timing of the kernel variants on all five configurations (not the headline)")
     ap.add_argument("--layers", default=None,
                     help="comma-separated layer names: run one instance of each (profiling runs)")
     args = ap.parse_args()
     if args.layers:
         global LAYER_FILTER
         LAYER_FILTER = set(args.layers.split(","))
-    if args.impl == "reference":
+    if args.suite:
+        run_suite(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
