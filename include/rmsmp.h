@@ -202,6 +202,34 @@ rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* layer, const void* d
                                          rmsmp_variant variant, void* stream);
 
 /*
+ * Many small-batch linear layers in one launch (Algorithm 1's forward line, layer after layer;
+ * Section 3.1: execution is "layer by layer on the same pieces of computing resource").  With a
+ * handful of tokens a layer is bound by reading its packed weights once, which takes a fraction
+ * of a microsecond -- less than a kernel launch -- so the layers are handed over together and one
+ * kernel streams all their weights.  Every item is computed exactly as rmsmp_gemm would (CUDA
+ * cores, codes expanded in registers).  Items must not write to memory another item reads
+ * (they run concurrently).
+ *   h_items   `count` host structures (1 <= count <= 65536), all linear layers.
+ *   d_table   device scratch of rmsmp_grouped_table_bytes(count) bytes, 16-byte aligned; the
+ *             library writes the problem table there (it must stay untouched until the work
+ *             queued by this call has finished).
+ * Errors: as rmsmp_gemm per item, BUFFER_TOO_SMALL for the table.
+ */
+typedef struct rmsmp_gemm_item {
+    const rmsmp_layer* layer;
+    const void* d_packed;
+    const int8_t* d_act;       /* [N][ld_act] */
+    int64_t N, ld_act;
+    float act_step;
+    float* d_out;
+    int64_t ld_out;
+    int32_t* d_acc;            /* optional */
+} rmsmp_gemm_item;
+rmsmp_status rmsmp_grouped_table_bytes(int count, size_t* bytes);
+rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
+                                void* d_table, size_t table_bytes, void* stream);
+
+/*
  * Workspace variant of the tensor-core path.  The expansion of the 4-bit / PoT codes to int8
  * (the GPU counterpart of routing rows to the per-scheme GEMM cores, Section 4.1) is done ONCE
  * per layer into caller-provided scratch memory instead of once per output tile in shared

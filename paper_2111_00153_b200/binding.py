@@ -30,7 +30,8 @@ EXPORTS = (
     "rmsmp_unpack_codes", "rmsmp_quantize_act", "rmsmp_gemm", "rmsmp_gemm_variant",
     "rmsmp_conv_implicit", "rmsmp_conv_implicit_variant", "rmsmp_last_device_status",
     "rmsmp_measure_mma_peak", "rmsmp_workspace_bytes", "rmsmp_expand_weights", "rmsmp_gemm_workspace",
-    "rmsmp_conv_implicit_workspace", "rmsmp_gemm_builtin_scratch",
+    "rmsmp_conv_implicit_workspace", "rmsmp_gemm_builtin_scratch", "rmsmp_grouped_table_bytes",
+    "rmsmp_gemm_grouped",
 )
 
 
@@ -50,6 +51,14 @@ class rmsmp_layer(C.Structure):
     @property
     def K(self) -> int:
         return self.Cin * self.kh * self.kw
+
+
+class rmsmp_gemm_item(C.Structure):
+    _fields_ = [
+        ("layer", C.POINTER(rmsmp_layer)), ("d_packed", C.c_void_p), ("d_act", C.c_void_p),
+        ("N", C.c_int64), ("ld_act", C.c_int64), ("act_step", C.c_float),
+        ("d_out", C.c_void_p), ("ld_out", C.c_int64), ("d_acc", C.c_void_p),
+    ]
 
 
 class RmsmpError(RuntimeError):
@@ -94,6 +103,8 @@ def lib() -> C.CDLL:
         L.rmsmp_workspace_bytes.argtypes = [C.POINTER(rmsmp_layer), C.POINTER(C.c_size_t)]
         L.rmsmp_expand_weights.argtypes = [C.POINTER(rmsmp_layer), vp, vp, C.c_size_t, vp]
         L.rmsmp_gemm_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
+        L.rmsmp_grouped_table_bytes.argtypes = [i32, C.POINTER(C.c_size_t)]
+        L.rmsmp_gemm_grouped.argtypes = [C.POINTER(rmsmp_gemm_item), i32, i32, vp, C.c_size_t, vp]
         L.rmsmp_gemm_builtin_scratch.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
         L.rmsmp_conv_implicit_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
                                                     f32, vp, i32, vp, vp]
@@ -248,6 +259,33 @@ def rmsmp_gemm_builtin_scratch(layer, d_packed, d_act, N: int, ld_act: int, act_
     _check(lib().rmsmp_gemm_builtin_scratch(C.byref(layer), _dp(d_packed), _dp(d_act), N, ld_act,
                                             act_step, _dp(d_out), ld_out, out_layout, _dp(d_acc),
                                             _stream(stream)), "rmsmp_gemm_builtin_scratch")
+
+
+def rmsmp_grouped_table_bytes(count: int) -> int:
+    n = C.c_size_t(0)
+    _check(lib().rmsmp_grouped_table_bytes(count, C.byref(n)), "rmsmp_grouped_table_bytes")
+    return n.value
+
+
+def make_gemm_items(items):
+    """items: iterable of (layer, d_packed, d_act, N, ld_act, act_step, d_out, ld_out, d_acc|None)
+    -> ctypes array of rmsmp_gemm_item (keep the layers alive while it is in use)."""
+    items = list(items)
+    arr = (rmsmp_gemm_item * len(items))()
+    for k, (layer, pk, act, N, ld_act, step, out, ld_out, acc) in enumerate(items):
+        arr[k].layer = C.pointer(layer)
+        arr[k].d_packed = pk.data_ptr(); arr[k].d_act = act.data_ptr()
+        arr[k].N = N; arr[k].ld_act = ld_act; arr[k].act_step = step
+        arr[k].d_out = out.data_ptr(); arr[k].ld_out = ld_out
+        arr[k].d_acc = acc.data_ptr() if acc is not None else None
+    return arr
+
+
+def rmsmp_gemm_grouped(items_array, out_layout: int, d_table, table_bytes: int | None = None, stream=None):
+    if table_bytes is None:
+        table_bytes = d_table.numel() * d_table.element_size()
+    _check(lib().rmsmp_gemm_grouped(items_array, len(items_array), out_layout, _dp(d_table), table_bytes,
+                                    _stream(stream)), "rmsmp_gemm_grouped")
 
 
 def rmsmp_last_device_status(d_packed, stream=None) -> int:

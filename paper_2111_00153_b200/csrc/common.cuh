@@ -61,6 +61,9 @@ cudaError_t launch_quantize_act(const float* x, size_t count, float alpha, int k
                                 cudaStream_t st);
 cudaError_t launch_simple(const Problem& p, cudaStream_t st);
 cudaError_t launch_simt(const Problem& p, bool shiftadd, cudaStream_t st);
+size_t grouped_table_bytes(int count);
+int grouped_fill_table(const Problem* probs, int count, uint8_t* h_table);
+cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t total, int nt, cudaStream_t st);
 // returns false if the tensor variant cannot run this problem (alignment / shape)
 bool tensor_supported(const Problem& p);
 rmsmp_status launch_tensor(const Problem& p, cudaStream_t st);

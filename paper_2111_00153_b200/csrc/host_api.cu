@@ -365,6 +365,62 @@ static rmsmp_status gemm_impl(const rmsmp_layer* L, const void* d_packed, const 
     return dispatch(p, variant, static_cast<cudaStream_t>(stream));
 }
 
+rmsmp_status rmsmp_grouped_table_bytes(int count, size_t* bytes)
+{
+    if (!bytes) return RMSMP_ERR_NULL;
+    if (count < 1 || count > 65536) return RMSMP_ERR_SHAPE;
+    *bytes = (grouped_table_bytes(count) + 255) / 256 * 256;
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
+                                void* d_table, size_t table_bytes, void* stream)
+{
+    if (!h_items || !d_table) return RMSMP_ERR_NULL;
+    if (count < 1 || count > 65536) return RMSMP_ERR_SHAPE;
+    if (out_layout != RMSMP_OUT_NM && out_layout != RMSMP_OUT_MN) return RMSMP_ERR_SHAPE;
+    if (table_bytes < grouped_table_bytes(count)) return RMSMP_ERR_BUFFER_TOO_SMALL;
+    if (!aligned16(d_table)) return RMSMP_ERR_ALIGN;
+    std::vector<Problem> probs((size_t)count);
+    for (int i = 0; i < count; ++i) {
+        const rmsmp_gemm_item& it = h_items[i];
+        const rmsmp_layer* L = it.layer;
+        if (!L || !it.d_packed || !it.d_act || !it.d_out) return RMSMP_ERR_NULL;
+        if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+        if (L->kh != 1 || L->kw != 1) return RMSMP_ERR_SHAPE;
+        if (it.N < 1 || it.N > (int64_t)1 << 31 || it.ld_act < L->Cin) return RMSMP_ERR_SHAPE;
+        if (it.ld_out < (out_layout == RMSMP_OUT_NM ? (int64_t)L->M : it.N)) return RMSMP_ERR_SHAPE;
+        if (!std::isfinite(it.act_step)) return RMSMP_ERR_SCALE;
+        if (!aligned16(it.d_act) || !aligned16(it.d_out) || (it.d_acc && !aligned16(it.d_acc)) || (it.ld_act & 15) ||
+            (reinterpret_cast<uintptr_t>(it.d_packed) & 255))
+            return RMSMP_ERR_ALIGN;
+        Problem& p = probs[(size_t)i];
+        fill_problem(p, L, it.d_packed);
+        p.act = it.d_act;
+        p.B = (int)std::min<int64_t>(it.N, 0x7fffffff); p.H = 1; p.W = 1; p.Ho = 1; p.Wo = 1; p.stride = 1; p.pad = 0;
+        p.pix_pitch = it.ld_act; p.N = it.N;
+        p.act_step = it.act_step; p.out = it.d_out; p.acc = it.d_acc; p.ld_out = it.ld_out;
+        p.out_mn = (out_layout == RMSMP_OUT_MN);
+    }
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    std::vector<uint8_t> table(grouped_table_bytes(count));
+    const int nt = grouped_fill_table(probs.data(), count, table.data());
+    int64_t total = 0;
+    std::memcpy(&total, table.data() + 8, sizeof(total));      // GroupedTable::total
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!staged_upload(d_table, table.data(), table.size(), st) &&
+        cudaMemcpyAsync(d_table, table.data(), table.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    if (launch_grouped(static_cast<const uint8_t*>(d_table), table.size(), total, nt, st) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return RMSMP_OK;
+}
+
 rmsmp_status rmsmp_gemm_variant(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act,
                                 int64_t N, int64_t ld_act, float act_step, float* d_out,
                                 int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,

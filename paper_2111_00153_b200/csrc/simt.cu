@@ -1,6 +1,7 @@
 // CUDA-core variants of the contraction: a one-thread-per-output cross-check kernel and a
 // row-per-warp kernel (integer dot products on codes expanded in registers, or -- for PoT
 // rows -- shifts and adds without a multiplier).
+#include <cstring>
 #include "common.cuh"
 #include "decode.cuh"
 
@@ -191,6 +192,232 @@ cudaError_t launch_simt(const Problem& p, bool shiftadd, cudaStream_t st)
     if (blocks > 148 * 8) blocks = 148 * 8;
     if (shiftadd) rowwarp_kernel<true><<<(unsigned)blocks, 256, 0, st>>>(p);
     else rowwarp_kernel<false><<<(unsigned)blocks, 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ grouped small-batch launch
+// Many weight-bound linear layers (a few tokens each) in ONE launch: with one launch per layer
+// the few hundred nanoseconds the weights need at HBM speed disappear behind launch latency.
+// The table in device memory holds the problems and the running count of work items; a work
+// item is (problem, up to RW consecutive packed rows of ONE kind, group of NT tokens), so the
+// row loop of an item has no per-row branches.  A warp keeps the 16-byte chunks of its RW rows
+// in flight together, so enough bytes are outstanding per SM to stream the packed weights at
+// memory speed.  Each block first copies the table to shared memory (when it fits), which takes
+// the table look-ups out of the dependent-load chain in front of every item's weight loads.
+
+struct GroupedTable {          // device layout: header, cum[count + 1], then Problem[count] at `prob_off`
+    int32_t count;
+    int32_t prob_off;          // bytes from the table start
+    int64_t total;             // work items
+    int32_t bytes;             // whole table
+    int32_t pad;
+};
+
+constexpr int kGroupedSmemMax = 96 * 1024;
+
+__host__ __device__ inline int grouped_rw(int kind, int nt)
+{
+    if (nt == 1) return kind == kFixed8 ? 4 : 8;
+    return 2;
+}
+
+template <int KIND>
+__device__ __forceinline__ void grouped_expand(const uint4& lo, const uint4& hi, uint32_t wv[8])
+{
+    if (KIND == kFixed8) {
+        wv[0] = lo.x; wv[1] = lo.y; wv[2] = lo.z; wv[3] = lo.w;
+        wv[4] = hi.x; wv[5] = hi.y; wv[6] = hi.z; wv[7] = hi.w;
+    } else if (KIND == kPoT4) {
+        expand_pot_chunk(lo, wv);
+    } else {
+        expand_fixed4_chunk_x16(lo, wv);
+    }
+}
+
+template <int KIND, int NT, int RW>
+__device__ __forceinline__ void grouped_rows(const Problem& p, int pr0, int nrows, int64_t n0, int lane)
+{
+    const int n4 = p.nP + p.nF4;
+    const int nchunks = p.Cp >> 5;                           // linear layers: one tap
+    const size_t pitch = (KIND == kFixed8) ? (size_t)p.Kp : (size_t)(p.Kp >> 1);
+    const uint8_t* base = (KIND == kFixed8) ? p.q8 + (size_t)(pr0 - n4) * pitch : p.q4 + (size_t)pr0 * pitch;
+    // Lane r fetches row r's original index and scale now, so that these two dependent loads
+    // overlap the weight stream instead of following it.
+    int row_m = 0;
+    float row_c = 0.0f;
+    if (lane < nrows) {
+        row_m = p.perm[pr0 + lane];
+        row_c = __fmul_rn(p.wstep[row_m], p.act_step);
+    }
+    int acc[RW][NT];
+#pragma unroll
+    for (int r = 0; r < RW; ++r)
+#pragma unroll
+        for (int t = 0; t < NT; ++t) acc[r][t] = 0;
+    for (int ch = lane; ch < nchunks; ch += 32) {
+        const int kp = ch << 5;
+        const size_t off = (KIND == kFixed8) ? (size_t)kp : (size_t)(kp >> 1);
+        uint4 raw[RW], raw2[KIND == kFixed8 ? RW : 1];
+#pragma unroll
+        for (int r = 0; r < RW; ++r) {                       // all rows' loads in flight together
+            const int rr = r < nrows ? r : nrows - 1;        // rows past the item's end repeat its last one
+            const uint4* src = reinterpret_cast<const uint4*>(base + (size_t)rr * pitch + off);
+            raw[r] = __ldcs(src);
+            if (KIND == kFixed8) raw2[r] = __ldcs(src + 1);
+        }
+        const bool full = (kp + 32 <= p.Cin);
+        // One token: its codes are loaded once and each row is expanded right before its dot
+        // product.  Several tokens: all rows are expanded first, then tokens stream through.
+        uint32_t wv[NT == 1 ? 1 : RW][8];
+        if (NT > 1) {
+#pragma unroll
+            for (int r = 0; r < RW; ++r) grouped_expand<KIND>(raw[r], raw2[KIND == kFixed8 ? r : 0], wv[NT == 1 ? 0 : r]);
+        }
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+            const int64_t n = (n0 + t < p.N) ? n0 + t : p.N - 1;
+            const int8_t* ap = p.act + n * p.pix_pitch + kp;
+            uint32_t a[8];
+            if (full) {
+                const uint4 lo = __ldg(reinterpret_cast<const uint4*>(ap)), hi = __ldg(reinterpret_cast<const uint4*>(ap) + 1);
+                a[0] = lo.x; a[1] = lo.y; a[2] = lo.z; a[3] = lo.w;
+                a[4] = hi.x; a[5] = hi.y; a[6] = hi.z; a[7] = hi.w;
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    uint32_t v = 0;
+#pragma unroll
+                    for (int bb = 0; bb < 4; ++bb)
+                        if (kp + q * 4 + bb < p.Cin) v |= (uint32_t)(uint8_t)ap[q * 4 + bb] << (8 * bb);
+                    a[q] = v;
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < RW; ++r) {
+                if (NT == 1) {
+                    grouped_expand<KIND>(raw[r], raw2[KIND == kFixed8 ? r : 0], wv[0]);
+                    acc[r][t] = dot32(wv[0], a, acc[r][t]);
+                } else {
+                    acc[r][t] = dot32(wv[NT == 1 ? 0 : r], a, acc[r][t]);
+                }
+            }
+        }
+    }
+    // Lane r*NT + t finishes element (row r, token t) with the row data lane r fetched up front.
+    int mine = 0;
+#pragma unroll
+    for (int r = 0; r < RW; ++r)
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+            int v = __reduce_add_sync(0xffffffffu, acc[r][t]);
+            if (KIND == kFixed4) v >>= 4;                    // the Fixed-4 codes were expanded as 16 * value
+            if (lane == r * NT + t) mine = v;
+        }
+    static_assert(RW * NT <= 32, "one lane per element of a work item");
+    const int er = lane / NT, et = lane % NT;
+    const int m = __shfl_sync(0xffffffffu, row_m, er & 31);
+    const float c = __shfl_sync(0xffffffffu, row_c, er & 31);
+    if (er < nrows && n0 + et < p.N) {
+        const int64_t n = n0 + et;
+        const int64_t o = p.out_mn ? (int64_t)m * p.ld_out + n : n * p.ld_out + m;
+        p.out[o] = __fmul_rn(__int2float_rn(mine), c);
+        if (p.acc) p.acc[o] = mine;
+    }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(256, 2) grouped_kernel(const uint8_t* __restrict__ gtable, int use_smem)
+{
+    extern __shared__ __align__(16) uint8_t s_table[];
+    const uint8_t* table = gtable;
+    if (use_smem) {
+        const int n16 = reinterpret_cast<const GroupedTable*>(gtable)->bytes >> 4;
+        for (int i = threadIdx.x; i < n16; i += blockDim.x)
+            reinterpret_cast<uint4*>(s_table)[i] = __ldg(reinterpret_cast<const uint4*>(gtable) + i);
+        __syncthreads();
+        table = s_table;
+    }
+    const GroupedTable* hdr = reinterpret_cast<const GroupedTable*>(table);
+    const int64_t* cum = reinterpret_cast<const int64_t*>(table + sizeof(GroupedTable));
+    const Problem* probs = reinterpret_cast<const Problem*>(table + hdr->prob_off);
+    constexpr int RW4 = (NT == 1) ? 8 : 2, RW8 = (NT == 1) ? 4 : 2;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t total = hdr->total;
+    int pi = 0;
+    for (int64_t w = warp0; w < total; w += nwarps) {
+        while (w >= cum[pi + 1]) ++pi;
+        const Problem& p = probs[pi];
+        const int64_t local = w - cum[pi];
+        const int iP = (p.nP + RW4 - 1) / RW4, iF = (p.nF4 + RW4 - 1) / RW4, i8 = (p.n8 + RW8 - 1) / RW8;
+        const int ipg = iP + iF + i8;
+        const int li = (int)(local % ipg);
+        const int64_t n0 = (local / ipg) * NT;
+        if (li < iP) {
+            const int r0 = li * RW4;
+            grouped_rows<kPoT4, NT, RW4>(p, r0, min(RW4, p.nP - r0), n0, lane);
+        } else if (li < iP + iF) {
+            const int r0 = (li - iP) * RW4;
+            grouped_rows<kFixed4, NT, RW4>(p, p.nP + r0, min(RW4, p.nF4 - r0), n0, lane);
+        } else {
+            const int r0 = (li - iP - iF) * RW8;
+            grouped_rows<kFixed8, NT, RW8>(p, p.nP + p.nF4 + r0, min(RW8, p.n8 - r0), n0, lane);
+        }
+    }
+}
+
+size_t grouped_table_bytes(int count)
+{
+    size_t off = sizeof(GroupedTable) + sizeof(int64_t) * (size_t)(count + 1);
+    off = (off + 15) / 16 * 16;
+    return (off + sizeof(Problem) * (size_t)count + 15) / 16 * 16;
+}
+
+// Fills `h_table` (grouped_table_bytes(count) bytes) from the problems; returns the token group size.
+int grouped_fill_table(const Problem* probs, int count, uint8_t* h_table)
+{
+    int64_t maxN = 1;
+    for (int i = 0; i < count; ++i) maxN = probs[i].N > maxN ? probs[i].N : maxN;
+    const int nt = (maxN == 1) ? 1 : kTok;
+    const int rw4 = grouped_rw(kPoT4, nt), rw8 = grouped_rw(kFixed8, nt);
+    memset(h_table, 0, grouped_table_bytes(count));
+    GroupedTable* hdr = reinterpret_cast<GroupedTable*>(h_table);
+    int64_t* cum = reinterpret_cast<int64_t*>(h_table + sizeof(GroupedTable));
+    size_t off = sizeof(GroupedTable) + sizeof(int64_t) * (size_t)(count + 1);
+    off = (off + 15) / 16 * 16;
+    hdr->count = count;
+    hdr->prob_off = (int32_t)off;
+    hdr->bytes = (int32_t)grouped_table_bytes(count);
+    cum[0] = 0;
+    for (int i = 0; i < count; ++i) {
+        const Problem& q = probs[i];
+        const int64_t ipg = (q.nP + rw4 - 1) / rw4 + (q.nF4 + rw4 - 1) / rw4 + (q.n8 + rw8 - 1) / rw8;
+        cum[i + 1] = cum[i] + ipg * ((q.N + nt - 1) / nt);
+    }
+    hdr->total = cum[count];
+    memcpy(h_table + off, probs, sizeof(Problem) * (size_t)count);
+    return nt;
+}
+
+cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t total, int nt, cudaStream_t st)
+{
+    int64_t blocks = (total + 7) / 8;
+    if (blocks > 148 * 2 * 4) blocks = 148 * 2 * 4;
+    if (blocks < 1) blocks = 1;
+    const int use_smem = table_bytes <= (size_t)kGroupedSmemMax;
+    const size_t smem = use_smem ? table_bytes : 0;
+    static bool attr_done[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(grouped_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupedSmemMax);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(grouped_kernel<kTok>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupedSmemMax);
+        if (e != cudaSuccess) return e;
+        attr_done[dev] = true;
+    }
+    if (nt == 1) grouped_kernel<1><<<(unsigned)blocks, 256, smem, st>>>(d_table, use_smem);
+    else grouped_kernel<kTok><<<(unsigned)blocks, 256, smem, st>>>(d_table, use_smem);
     return cudaGetLastError();
 }
 

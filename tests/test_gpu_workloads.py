@@ -169,3 +169,38 @@ def test_config5_bert_large_small_batch(name, M, K, N, ratio):
         y, acc = Hn.gemm(layer, d_packed, act, 0.05, variant)
         assert np.array_equal(acc, acc_ref)
         assert np.array_equal(y.view(np.uint32), y_ref.view(np.uint32))
+
+
+# ------------------------------------------------------------------ config 5, grouped: many layers, one launch
+
+@pytest.mark.parametrize("N", [1, 8, 5])
+def test_config5_grouped_launch_matches_oracle(N):
+    import torch
+    shapes = [(1024, 1024), (4096, 1024), (1024, 4096), (130, 96), (64, 40)]
+    keep, items, refs = [], [], []
+    for i, (M, K) in enumerate(shapes):
+        g = synth.rng(5, 900 + i + N)
+        W = synth.weights_normal(g, (M, K))
+        ratio = synth.RATIO_SWEEP[i % 4]
+        scheme, bits = O.assign_rows(W, ratio)
+        alpha = synth.alpha_rows(W)
+        act = synth.act_codes_uniform(g, (N, K))
+        layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+        ld = (K + 15) // 16 * 16
+        a = torch.zeros((N, ld), dtype=torch.int8, device="cuda")
+        a[:, :K] = torch.from_numpy(act).cuda()
+        y = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+        acc = torch.full((N, M), -5, dtype=torch.int32, device="cuda")
+        step = float(np.float32(0.01 * (i + 1)))
+        keep.append((layer, d_packed, a, y, acc))
+        items.append((layer, d_packed, a, N, ld, step, y, M, acc))
+        v_ref, wstep = O.quantize_rows(W, scheme, bits, alpha)
+        acc_ref = O.matmul(v_ref, act)
+        refs.append((acc_ref, _expected(acc_ref, wstep, np.float32(step))))
+    arr = R.make_gemm_items(items)
+    table = torch.empty(R.rmsmp_grouped_table_bytes(len(items)), dtype=torch.uint8, device="cuda")
+    R.rmsmp_gemm_grouped(arr, R.OUT_NM, table)
+    torch.cuda.synchronize()
+    for (layer, d_packed, a, y, acc), (acc_ref, y_ref) in zip(keep, refs):
+        assert np.array_equal(acc.cpu().numpy(), acc_ref)
+        assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
