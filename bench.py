@@ -299,7 +299,8 @@ def run_ours(args):
         "gpu_launches": args.steps * len(layers) * (4 if use_ws else 3),
         "roofline": {"bound": "hbm", "kernel": "tensor_kernel (conv_implicit)", "achieved": achieved_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved_gbs / peaks["hbm_gbs"],
-                     "peak_source": peak_src, "traffic": TRAFFIC_PER_STEP_BYTES,
+                     "peak_source": peak_src,
+                     "traffic": TRAFFIC_PER_STEP_BYTES if (batch == BATCH and use_ws and not args.layers) else None,
                      "algorithmic_bytes_per_step": float(alg.sum()), "kernel_ms_per_step": conv_total_ms,
                      "kernel_tops": ops_step / (conv_total_ms * 1e-3) / 1e12},
         "per_layer": [{"name": h["L"].name, "M": h["L"].M, "K": h["L"].K, "N": d["N"], "ms": float(ms),
@@ -313,9 +314,10 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# dram bytes (read + write) of the convolution kernels of one step, from an ncu capture; None
-# until measured for the current kernel.
-TRAFFIC_PER_STEP_BYTES = None
+# dram bytes (read + write) of the 19 convolution launches of one step at batch 256, from an ncu
+# capture of this kernel (profiles/bench_resnet18_stack_launch_list.md); reported only for that
+# configuration.  Set back to None whenever tensor_kernel changes.
+TRAFFIC_PER_STEP_BYTES = 1257.3e6
 
 
 def load_peaks():

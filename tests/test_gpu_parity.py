@@ -193,6 +193,9 @@ CONV_CASES = [
     (140, 256, 3, 1, 1, 5, 7, 7),     # several images per tile, ragged last tile
     (20, 20, 3, 1, 1, 1, 6, 6),       # Cin not a multiple of 16: CUDA-core variants only
     (64, 64, 3, 1, 1, 1, 56, 56),
+    (200, 64, 2, 1, 0, 2, 9, 9),      # 64-byte pixels, even tap count, two row blocks (weights through the ring)
+    (96, 64, 3, 2, 1, 3, 7, 7),       # 64-byte pixels, several images per tile, stride 2
+    (64, 48, 1, 1, 0, 2, 12, 12),     # 64-byte pixels, one tap
 ]
 
 
