@@ -157,7 +157,8 @@ rmsmp_status rmsmp_unpack_codes(const rmsmp_layer* layer, const void* d_packed,
  * One clip value per tensor.  U4: a = round_half_even(clip(x/alpha_a, 0, 1) * 15), step
  * alpha_a/15.  S4: Fixed-4 of Eq. 1 with alpha_a, step alpha_a/7.  d_X: `count` floats;
  * d_codes: `count` int8 (one code per byte).  *h_act_step receives the step (host, may be
- * NULL).  Pointers need only their natural alignment.  Errors: NULL, SHAPE, SCALE, ARCH, CUDA.
+ * NULL).  Infinite inputs clip like any other value; the code of a NaN input is unspecified.
+ * Pointers need only their natural alignment.  Errors: NULL, SHAPE, SCALE, ARCH, CUDA.
  */
 rmsmp_status rmsmp_quantize_act(const float* d_X, size_t count, float alpha_a,
                                 rmsmp_act_kind kind, int8_t* d_codes, float* h_act_step,

@@ -241,7 +241,13 @@ cudaError_t launch_expand(const rmsmp_layer& L, const uint8_t* blob, int8_t* wex
 }
 
 // ------------------------------------------------------------------ activation quantizer
-// Pure streaming kernel: 16 bytes of fp32 in, 4 code bytes out per thread step.
+// Pure streaming kernel.  The code is rint(clip(x / alpha) * Q) with ONE correctly rounded fp32
+// division; that division costs more issue slots than the memory system leaves time for, so the
+// vector path first forms the code from x * (1 / alpha) and keeps it only when the scaled value
+// is not within 0.001 of a rounding boundary (k + 0.5), where the two ways of computing x / alpha
+// (relative difference < 2^-22) cannot round to different integers; the few values that are
+// close to a boundary, and NaNs, take the division.  The results are those of act_code() in
+// every case.
 
 __device__ __forceinline__ int act_code(float x, float alpha, int kind)
 {
@@ -254,6 +260,45 @@ __device__ __forceinline__ int act_code(float x, float alpha, int kind)
     return __float2int_rn(__fmul_rn(t, 7.0f));
 }
 
+struct ActFast {
+    float r, lo, q;        // 1 / alpha, lower clip, levels per unit
+    bool ok;               // alpha is far from the ends of the fp32 range, so r is accurate
+};
+
+__device__ __forceinline__ ActFast act_fast_setup(float alpha, int kind)
+{
+    ActFast f;
+    f.r = __frcp_rn(alpha);
+    f.lo = (kind == RMSMP_ACT_U4) ? 0.0f : -1.0f;
+    f.q = (kind == RMSMP_ACT_U4) ? 15.0f : 7.0f;
+    f.ok = (alpha > 1e-30f) && (alpha < 1e30f);
+    return f;
+}
+
+// Code of x in the low byte of the result; sets `redo` when the division has to decide.
+__device__ __forceinline__ uint32_t act_code_fast(float x, const ActFast& f, bool& redo)
+{
+    const float kMagic = 12582912.0f;                       // 1.5 * 2^23: adding it rounds to an integer, half to even
+    float t = __fmul_rn(x, f.r);
+    t = fminf(fmaxf(t, f.lo), 1.0f);
+    const float u = __fmul_rn(t, f.q);
+    const float s = __fadd_rn(u, kMagic);
+    const float c = __fsub_rn(s, kMagic);
+    redo = redo || !(fabsf(__fsub_rn(u, c)) <= 0.499f);       // also true for NaN
+    return __float_as_uint(s);                               // low byte = the integer, two's complement
+}
+
+__device__ __forceinline__ uint32_t act_codes4(const float4& v, float alpha, int kind, const ActFast& f)
+{
+    bool redo = !f.ok;
+    const uint32_t a = act_code_fast(v.x, f, redo), b = act_code_fast(v.y, f, redo),
+                   c = act_code_fast(v.z, f, redo), d = act_code_fast(v.w, f, redo);
+    if (redo)
+        return (uint32_t)(act_code(v.x, alpha, kind) & 0xFF) | ((uint32_t)(act_code(v.y, alpha, kind) & 0xFF) << 8) |
+               ((uint32_t)(act_code(v.z, alpha, kind) & 0xFF) << 16) | ((uint32_t)(act_code(v.w, alpha, kind) & 0xFF) << 24);
+    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
+
 __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restrict__ x, size_t count,
                                                            float alpha, int kind,
                                                            int8_t* __restrict__ codes, int vec)
@@ -261,27 +306,24 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restri
     const size_t tid = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
     const size_t nthr = (size_t)gridDim.x * blockDim.x;
     if (vec) {
-        // 32 values per thread step: eight 128-bit loads in flight, then two 128-bit stores
+        // A warp takes 1024 consecutive values per step: eight 128-bit loads per lane, each
+        // instruction covering 512 contiguous bytes, then eight 32-bit stores of 128 contiguous
+        // bytes each.  The remaining 16-value groups follow one lane at a time.
         const size_t n16 = count / 16;
-        const size_t n32 = count / 32;
-        for (size_t i = tid; i < n32; i += nthr) {
-            const float4* src = reinterpret_cast<const float4*>(x) + i * 8;
+        const size_t n1024 = count / 1024;
+        const int lane = threadIdx.x & 31;
+        const size_t warp = tid >> 5, nwarp = nthr >> 5;
+        const ActFast fast = act_fast_setup(alpha, kind);
+        for (size_t i = warp; i < n1024; i += nwarp) {
+            const float4* src = reinterpret_cast<const float4*>(x) + i * 256 + lane;
             float4 v[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = __ldcs(src + j);
-            uint32_t w[8];
+            for (int j = 0; j < 8; ++j) v[j] = __ldcs(src + j * 32);
+            uint32_t* dst = reinterpret_cast<uint32_t*>(codes) + i * 256 + lane;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                w[j] = (uint32_t)(act_code(v[j].x, alpha, kind) & 0xFF) |
-                       ((uint32_t)(act_code(v[j].y, alpha, kind) & 0xFF) << 8) |
-                       ((uint32_t)(act_code(v[j].z, alpha, kind) & 0xFF) << 16) |
-                       ((uint32_t)(act_code(v[j].w, alpha, kind) & 0xFF) << 24);
-            uint4* dst = reinterpret_cast<uint4*>(codes) + i * 2;
-            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            for (int j = 0; j < 8; ++j) __stcs(dst + j * 32, act_codes4(v[j], alpha, kind, fast));
         }
-        if ((n16 & 1) && tid == 0) {              // one 16-value group left over
-            const size_t i = n16 - 1;
+        for (size_t i = n1024 * 64 + tid; i < n16; i += nthr) {
             const float4* src = reinterpret_cast<const float4*>(x) + i * 4;
             uint32_t w[4];
 #pragma unroll
@@ -304,7 +346,7 @@ cudaError_t launch_quantize_act(const float* x, size_t count, float alpha, int k
                                 cudaStream_t st)
 {
     int vec = ((reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(codes) & 15) == 0);
-    size_t steps = vec ? (count + 31) / 32 : count;
+    size_t steps = vec ? (count + 31) / 32 : count;      // the vector path handles 32 values per thread and step
     size_t blocks = (steps + 255) / 256;
     const size_t cap = 148 * 32;
     if (blocks > cap) blocks = cap;

@@ -108,6 +108,33 @@ def test_quantize_act(count, kind):
     assert step == s_ref
 
 
+@pytest.mark.parametrize("alpha", [3.0, 2.9999998, 1.0, 1e-3, 7.3e5, 1e-35, 1e33])
+@pytest.mark.parametrize("kind", [R.ACT_U4, R.ACT_S4])
+def test_quantize_act_on_rounding_boundaries(alpha, kind):
+    # Values on and a few ulps around every rounding boundary (k + 0.5) * alpha / Q and every level,
+    # around the clip points, plus specials, repeated until the warp-wide vector path is used.
+    # The code near a boundary depends on the single correctly rounded division x / alpha.
+    Q = 15 if kind == R.ACT_U4 else 7
+    a32 = np.float32(alpha)
+    ks = np.arange(-2 * Q - 3, 2 * Q + 4, dtype=np.float64) / 2.0          # levels and half-levels, beyond the clips
+    centre = (ks * np.float64(a32) / Q).astype(np.float32)
+    pts = [centre]
+    for d in range(1, 5):
+        up, dn = centre.copy(), centre.copy()
+        for _ in range(d):
+            up = np.nextafter(up, np.float32(np.inf)); dn = np.nextafter(dn, np.float32(-np.inf))
+        pts += [up, dn]
+    special = np.array([0.0, -0.0, np.inf, -np.inf, np.finfo(np.float32).tiny, 1e-45, -1e-45,
+                        np.finfo(np.float32).max], dtype=np.float32)
+    x = np.concatenate(pts + [special]).astype(np.float32)
+    g = synth.rng(72, 991)
+    x = np.concatenate([x, g.permutation(np.tile(x, 8))])                  # > 4096 values, mixed inside each warp step
+    codes, step = Hn.quantize_act(x, float(a32), kind)
+    c_ref, s_ref = O.quantize_act(x, float(a32), kind)
+    assert np.array_equal(codes, c_ref)
+    assert step == s_ref
+
+
 # ------------------------------------------------------------------ linear layer
 
 LIN_CASES = [
