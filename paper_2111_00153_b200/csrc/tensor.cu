@@ -72,6 +72,10 @@ struct TensorCfg {
     int a_bytes, b_bytes;  // one A / B stage
     int ares;              // 1 (pre mode, one row block, small K): the expanded weights of all k-blocks are loaded once
                            //    per CTA and stay in shared memory; only activation boxes flow through a ring
+    int m2;                // 1 (pre mode, even number of row blocks): a tile covers TWO row blocks.  Both use the same
+                           //    activation stage, so a k-block brings 64 KB for eight MMAs instead of 48 KB for four;
+                           //    the two accumulators take the two halves of tensor memory
+    int nbt;               // row-block groups per pixel tile: nblocks, or nblocks / 2
     uint32_t smem_bytes;
 };
 
@@ -275,6 +279,8 @@ __device__ __forceinline__ void expand_task(uint32_t meta, uint32_t raw_stage, u
 
 // ------------------------------------------------------------------ the kernel
 
+// kM2: a tile covers two row blocks (TensorCfg::m2), compiled separately so that the common form keeps its registers.
+template <int kM2>
 __global__ void __launch_bounds__(kThreads, 1)
 tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps maps)
 {
@@ -348,8 +354,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
             uint32_t s = 0, ph = 0;
             bool ok = true;
             for (int64_t tile = first; tile < cfg.ntiles && ok; tile += step) {
-                const int64_t nt = tile / p.nblocks;
-                const int blk = (int)(tile - nt * p.nblocks);
+                const int64_t nt = tile / cfg.nbt;
+                const int blk = (int)(tile - nt * cfg.nbt) << kM2;
                 int b0, h0;
                 if (cfg.tiles_per_image) { b0 = (int)(nt / cfg.tiles_per_image); h0 = (int)(nt % cfg.tiles_per_image) * cfg.th; }
                 else { b0 = (int)(nt * cfg.tb); h0 = 0; }
@@ -468,8 +474,10 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
             uint32_t sa = 0, phA = 0, sb = 0, phB = 0, it = 0;
             bool have_a = !cfg.ares || my_tiles == 0 || mbar_wait(bar_fullA, 0, abort_flag);
             for (int64_t tile = first; tile < cfg.ntiles && have_a && !*abort_flag; tile += step, ++it) {
-                const uint32_t ab = it & 1;
-                if (!mbar_wait(bar_tempty + 8 * ab, ((it >> 1) & 1) ^ 1, abort_flag)) break;
+                // one accumulator per tile, alternating; or (two row blocks per tile) both, every tile
+                const uint32_t ab = kM2 ? 0u : (it & 1);
+                const uint32_t tpar = kM2 ? ((it & 1) ^ 1) : (((it >> 1) & 1) ^ 1);
+                if (!mbar_wait(bar_tempty + 8 * ab, tpar, abort_flag)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + ab * kTileN;
                 bool ok = true;
@@ -483,6 +491,16 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                                    bd = smem_desc_kmajor(sB + sb * cfg.b_bytes, cfg.bk);
                     for (int ks = 0; ks < ksteps; ++ks)
                         mma_i8(d_tmem, ad + 2 * ks, bd + 2 * ks, cfg.idesc, (kb | ks) ? 1u : 0u);
+                    if (kM2) {
+                        // second row block: rows 128..255 of the weight stage, second accumulator
+                        if (kb == 0) {
+                            if (!mbar_wait(bar_tempty + 8, tpar, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                        }
+                        const uint64_t ad1 = ad + (kABytes >> 4);
+                        for (int ks = 0; ks < ksteps; ++ks)
+                            mma_i8(d_tmem + kTileN, ad1 + 2 * ks, bd + 2 * ks, cfg.idesc, (kb | ks) ? 1u : 0u);
+                    }
                     if (!cfg.ares) mma_commit(bar_emptyA + 8 * sa);
                     mma_commit(bar_emptyB + 8 * sb);
                     if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; }
@@ -491,6 +509,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 }
                 if (!ok) break;
                 mma_commit(bar_tfull + 8 * ab);
+                if (kM2) mma_commit(bar_tfull + 8);
             }
         }
     } else if (!cfg.pre && warp < 2 + kNumExpWarps) {
@@ -569,10 +588,14 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         const int cfirst = (cfg.dup && (quarter >> 1)) ? count_q(quarter & 1) + my_rank : my_rank;
         const uint32_t my_stage = sOut + (uint32_t)ew * (cfg.out_bufs * kWarpStage);
         uint32_t it = 0, stg_count = 0;
-        for (int64_t tile = first; tile < cfg.ntiles; tile += step, ++it) {
-            const uint32_t ab = it & 1;
-            const int blk = (int)(tile % p.nblocks);
-            const int64_t nt = tile / p.nblocks;
+        bool alive = true;
+        for (int64_t tile = first; tile < cfg.ntiles && alive; tile += step, ++it) {
+          // a tile is one row block (accumulators alternate between tiles), or two (one accumulator each)
+          for (int half = 0; half <= kM2; ++half) {
+            const uint32_t ab = kM2 ? (uint32_t)half : (it & 1);
+            const uint32_t tpar = kM2 ? (it & 1) : ((it >> 1) & 1);
+            const int64_t nt = tile / cfg.nbt;
+            const int blk = ((int)(tile - nt * cfg.nbt) << kM2) + half;
             int64_t n0;
             if (cfg.tiles_per_image) n0 = ((nt / cfg.tiles_per_image) * p.Ho + (nt % cfg.tiles_per_image) * cfg.th) * (int64_t)p.Wo;
             else n0 = nt * (int64_t)cfg.npix;
@@ -585,7 +608,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 scale = __fmul_rn(__ldg(p.wstep + m), p.act_step);
                 shift = (!cfg.pre && __ldg(p.kind + m) == kFixed4) ? 4 : 0;   // expanders store Fixed-4 codes as 16 * value
             }
-            if (!mbar_wait_warp(bar_tfull + 8 * ab, (it >> 1) & 1, abort_flag)) break;
+            if (!mbar_wait_warp(bar_tfull + 8 * ab, tpar, abort_flag)) { alive = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * kTileN;
             const int nchunks = (nvalid + 31) >> 5;
@@ -690,6 +713,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                     if (more2) tmem_ld_wait(va);
                 }
             }
+          }
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
@@ -728,6 +752,18 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) cudaGetLastError();
+        n = v > 0 ? v : 148;
+    }
+    return n;
+}
+
 bool plan(const Problem& p, TensorCfg& c)
 {
     if (p.pix_pitch % 16 != 0 || p.Cin % 16 != 0) return false;
@@ -753,6 +789,8 @@ bool plan(const Problem& p, TensorCfg& c)
     c.npix = c.tb * c.th * p.Wo;
     c.n_mma = (c.npix + 15) / 16 * 16;
     c.ntiles = c.ntiles_n * p.nblocks;
+    c.m2 = 0;
+    c.nbt = p.nblocks;
     c.pre = p.wexp ? 1 : 0;
     // 64-byte k-blocks when a 128-byte row would be at most half used by the (last) channel chunk
     c.bk = (c.pre && (p.Cin % 128 != 0) && (p.Cin % 128 <= 64)) ? 64 : 128;
@@ -781,6 +819,18 @@ bool plan(const Problem& p, TensorCfg& c)
             const int64_t left = kSmemLimit - (1024 + 64 * kMaxRing) - (int64_t)c.nkb * c.a_bytes -
                                  (int64_t)c.epi_warps * kWarpStage;
             c.nB = (int)std::min<int64_t>(kMaxRing, left / c.b_bytes);
+        }
+        // Two row blocks per tile pay when K is long (the two accumulators' epilogue is only half
+        // hidden behind the next tile's MMAs) and when the halved tile count does not cost more in
+        // idle SMs of the last wave than the ~20 % a double tile saves.
+        const int64_t sms = sm_count();
+        const int64_t waves1 = (c.ntiles + sms - 1) / sms, waves2 = (c.ntiles / 2 + sms - 1) / sms;
+        if (!c.ares && !c.dup && c.bk == 128 && p.nblocks % 2 == 0 && c.nkb >= 16 && 16 * waves2 < 10 * waves1) {
+            c.m2 = 1;
+            c.nbt = p.nblocks / 2;
+            c.ntiles = c.ntiles_n * c.nbt;
+            c.a_bytes = 2 * kABytes;
+            c.nA = 2; c.nB = 3;
         }
         c.smem_bytes = (uint32_t)(c.nA * c.a_bytes + c.nB * c.b_bytes + c.epi_warps * c.out_bufs * kWarpStage + 1024 +
                                   64 * kMaxRing);
@@ -845,7 +895,7 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
     if (p.wexp) {
         const cuuint64_t gd[2] = {(cuuint64_t)p.Kp, (cuuint64_t)p.M};
         const cuuint64_t gs[1] = {(cuuint64_t)p.Kp};
-        const cuuint32_t bx[2] = {(cuuint32_t)c.bk, (cuuint32_t)(c.dup ? kBlockRows / 2 : kBlockRows)};
+        const cuuint32_t bx[2] = {(cuuint32_t)c.bk, (cuuint32_t)(c.dup ? kBlockRows / 2 : (c.m2 ? 2 * kBlockRows : kBlockRows))};
         const cuuint32_t es[2] = {1, 1};
         if (enc(&mp.wexp, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(p.wexp), gd, gs, bx, es,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, c.bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
@@ -878,20 +928,18 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
         c.tma_store = ok ? 1 : 0;
     }
 
-    static int sm_count = 0;
     static bool attr_set = false;
     if (!attr_set) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (cudaFuncSetAttribute(tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tensor_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(tensor_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
             cudaGetLastError();
             return RMSMP_ERR_CUDA;
         }
         attr_set = true;
     }
-    const int grid = (int)std::min<int64_t>(c.ntiles, sm_count > 0 ? sm_count : 148);
-    tensor_kernel<<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
+    const int grid = (int)std::min<int64_t>(c.ntiles, sm_count());
+    if (c.m2) tensor_kernel<1><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
+    else tensor_kernel<0><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
     if (cudaGetLastError() != cudaSuccess) return RMSMP_ERR_CUDA;
     return RMSMP_OK;
 }

@@ -148,6 +148,7 @@ LIN_CASES = [
     (200, 48, 40, (0, 0, 100)),
     (150, 1000, 33, (100, 0, 0)),
     (257, 2304, 260, (60, 35, 5)),
+    (500, 640, 300, (60, 35, 5)),       # four row blocks: two per tile in the workspace variant, ragged last block
 ]
 
 

@@ -102,6 +102,33 @@ def test_config3_bert_base_linear(name, M, K):
         assert np.array_equal(y.cpu().numpy()[n_idx, m_idx].view(np.uint32), want.view(np.uint32))
 
 
+def test_two_row_blocks_per_tile_full():
+    """Long K, two row blocks and two waves of single-block tiles: the shape class for which the
+    workspace variant runs both row blocks of a tile against one activation stage.  Every
+    accumulator and output against the oracle; 19000 tokens leave a ragged last tile."""
+    import torch
+    M, K, N = 256, 2048, 19000
+    g = synth.rng(3, 77)
+    W = synth.weights_normal(g, (M, K))
+    c_ref = synth.act_codes_uniform(g, (N, K))
+    step = np.float32(0.0625)
+    scheme, bits = O.assign_rows(W, synth.RATIO_RMSMP1)
+    alpha = synth.alpha_rows(W)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    codes = torch.from_numpy(c_ref).cuda()
+    y = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+    acc = torch.empty((N, M), dtype=torch.int32, device="cuda")
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    R.rmsmp_gemm_workspace(layer, d_packed, ws, codes, N, K, float(step), y, M, R.OUT_NM, acc)
+    torch.cuda.synchronize()
+    assert R.rmsmp_last_device_status(d_packed) == R.OK
+    v_ref, wstep = O.quantize_rows(W, scheme, bits, alpha)
+    acc_ref = O.matmul(v_ref, c_ref)
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), _expected(acc_ref, wstep, step).view(np.uint32))
+
+
 # ------------------------------------------------------------------ config 4: the ResNet-18 stack
 
 @pytest.mark.parametrize("L", synth.resnet18_convs(), ids=lambda L: L.name)
