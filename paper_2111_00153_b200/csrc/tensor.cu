@@ -76,6 +76,9 @@ struct TensorCfg {
                            //    activation stage, so a k-block brings 64 KB for eight MMAs instead of 48 KB for four;
                            //    the two accumulators take the two halves of tensor memory
     int nbt;               // row-block groups per pixel tile: nblocks, or nblocks / 2
+    int tps;               // k-blocks per activation stage: 1, or 3 (resident weights, 64-byte k-blocks, 3-wide kernels):
+                           //    one barrier round trip then covers a whole kernel row instead of a single tap
+    int b_sub;             // bytes of one k-block inside an activation stage
     uint32_t smem_bytes;
 };
 
@@ -184,6 +187,21 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Same, with the descriptors given as 32-bit halves.  The MMA thread runs alone at a few cycles
+// per instruction, and its per-k-block instruction count shows directly in the kernel time, so
+// it keeps only the low words (address field) moving and leaves the high words constant.
+__device__ __forceinline__ void mma_i8_halves(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                              uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar)
@@ -364,6 +382,16 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 int tap = 0, cc = 0, ti = 0, tj = 0;
                 for (int kb = 0; kb < cfg.nkb; ++kb) {
                     if (!mbar_wait(bar_e + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
+                    if (pre_b_producer && cfg.tps > 1) {
+                        // one stage = the taps of one kernel row (one channel chunk per tap in this mode)
+                        mbar_arrive_expect_tx(bar_f + 8 * s, cfg.tps * cfg.tx_bytes);
+                        for (int t = 0; t < cfg.tps; ++t)
+                            tma_load_4d(sB + s * cfg.b_bytes + t * cfg.b_sub, &maps.act, bar_f + 8 * s, 0, tj + t - p.pad, y_base + ti, b0);
+                        ++ti;
+                        kb += cfg.tps - 1;
+                        if (++s == nring) { s = 0; ph ^= 1; }
+                        continue;
+                    }
                     if (pre_b_producer) {
                         mbar_arrive_expect_tx(bar_f + 8 * s, cfg.tx_bytes);
                         tma_load_4d(sB + s * cfg.b_bytes, &maps.act, bar_f + 8 * s, cc * cfg.bk, tj - p.pad, y_base + ti, b0);
@@ -472,6 +500,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         // ---------------------------------------------------------- MMA issuer
         if (lane == 0) {
             uint32_t sa = 0, phA = 0, sb = 0, phB = 0, it = 0;
+            const uint64_t desc_a0 = smem_desc_kmajor(sA, cfg.bk), desc_b0 = smem_desc_kmajor(sB, cfg.bk);
+            const uint32_t desc_lo0_a = (uint32_t)desc_a0, desc_lo0_b = (uint32_t)desc_b0, desc_hi = (uint32_t)(desc_a0 >> 32);
             bool have_a = !cfg.ares || my_tiles == 0 || mbar_wait(bar_fullA, 0, abort_flag);
             for (int64_t tile = first; tile < cfg.ntiles && have_a && !*abort_flag; tile += step, ++it) {
                 // one accumulator per tile, alternating; or (two row blocks per tile) both, every tile
@@ -482,30 +512,52 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 const uint32_t d_tmem = tmem_base + ab * kTileN;
                 bool ok = true;
                 int cc = 0;
-                for (int kb = 0; kb < cfg.nkb; ++kb) {
-                    if (!mbar_wait(bar_fullB + 8 * sb, phB, abort_flag) ||
-                        (!cfg.ares && !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag))) { ok = false; break; }
-                    tc_fence_after();
-                    const int ksteps = (cc == cfg.cpt - 1) ? cfg.last_ksteps : (cfg.bk >> 5);
-                    const uint64_t ad = smem_desc_kmajor(sA + (cfg.ares ? (uint32_t)kb : sa) * cfg.a_bytes, cfg.bk),
-                                   bd = smem_desc_kmajor(sB + sb * cfg.b_bytes, cfg.bk);
-                    for (int ks = 0; ks < ksteps; ++ks)
-                        mma_i8(d_tmem, ad + 2 * ks, bd + 2 * ks, cfg.idesc, (kb | ks) ? 1u : 0u);
-                    if (kM2) {
-                        // second row block: rows 128..255 of the weight stage, second accumulator
-                        if (kb == 0) {
-                            if (!mbar_wait(bar_tempty + 8, tpar, abort_flag)) { ok = false; break; }
-                            tc_fence_after();
+                if (cfg.tps > 1) {
+                    // resident weights, several k-blocks per activation stage (never with two row blocks)
+                    for (int kb = 0; kb < cfg.nkb; kb += cfg.tps) {
+                        if (!mbar_wait(bar_fullB + 8 * sb, phB, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        for (int t = 0; t < cfg.tps; ++t) {
+                            const uint64_t ad = smem_desc_kmajor(sA + (uint32_t)(kb + t) * cfg.a_bytes, cfg.bk),
+                                           bd = smem_desc_kmajor(sB + sb * cfg.b_bytes + t * cfg.b_sub, cfg.bk);
+                            for (int ks = 0; ks < cfg.last_ksteps; ++ks)
+                                mma_i8(d_tmem, ad + 2 * ks, bd + 2 * ks, cfg.idesc, (kb | t | ks) ? 1u : 0u);
                         }
-                        const uint64_t ad1 = ad + (kABytes >> 4);
-                        for (int ks = 0; ks < ksteps; ++ks)
-                            mma_i8(d_tmem + kTileN, ad1 + 2 * ks, bd + 2 * ks, cfg.idesc, (kb | ks) ? 1u : 0u);
+                        mma_commit(bar_emptyB + 8 * sb);
+                        if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; }
                     }
-                    if (!cfg.ares) mma_commit(bar_emptyA + 8 * sa);
-                    mma_commit(bar_emptyB + 8 * sb);
-                    if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; }
-                    if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; }
-                    if (++cc == cfg.cpt) cc = 0;
+                } else {
+                    const bool uniform = (cfg.last_ksteps == (cfg.bk >> 5));      // every k-block has the same depth
+                    const uint32_t a_step = (uint32_t)cfg.a_bytes >> 4, b_step = (uint32_t)cfg.b_bytes >> 4;
+                    uint32_t a_lo = cfg.ares ? desc_lo0_a : desc_lo0_a + sa * a_step;
+                    uint32_t b_lo = desc_lo0_b + sb * b_step;
+                    for (int kb = 0; kb < cfg.nkb; ++kb) {
+                        if (!mbar_wait(bar_fullB + 8 * sb, phB, abort_flag) ||
+                            (!cfg.ares && !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag))) { ok = false; break; }
+                        tc_fence_after();
+                        const int ksteps = (uniform || cc != cfg.cpt - 1) ? (cfg.bk >> 5) : cfg.last_ksteps;
+                        mma_i8_halves(d_tmem, a_lo, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
+                        for (int ks = 1; ks < ksteps; ++ks)
+                            mma_i8_halves(d_tmem, a_lo + 2 * ks, b_lo + 2 * ks, desc_hi, cfg.idesc, 1u);
+                        if (kM2) {
+                            // second row block: rows 128..255 of the weight stage, second accumulator
+                            if (kb == 0) {
+                                if (!mbar_wait(bar_tempty + 8, tpar, abort_flag)) { ok = false; break; }
+                                tc_fence_after();
+                            }
+                            const uint32_t a1 = a_lo + (kABytes >> 4);
+                            mma_i8_halves(d_tmem + kTileN, a1, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
+                            for (int ks = 1; ks < ksteps; ++ks)
+                                mma_i8_halves(d_tmem + kTileN, a1 + 2 * ks, b_lo + 2 * ks, desc_hi, cfg.idesc, 1u);
+                        }
+                        if (!cfg.ares) mma_commit(bar_emptyA + 8 * sa);
+                        mma_commit(bar_emptyB + 8 * sb);
+                        a_lo += a_step;
+                        b_lo += b_step;
+                        if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; if (!cfg.ares) a_lo = desc_lo0_a; }
+                        if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; b_lo = desc_lo0_b; }
+                        if (!uniform && ++cc == cfg.cpt) cc = 0;
+                    }
                 }
                 if (!ok) break;
                 mma_commit(bar_tfull + 8 * ab);
@@ -791,6 +843,8 @@ bool plan(const Problem& p, TensorCfg& c)
     c.ntiles = c.ntiles_n * p.nblocks;
     c.m2 = 0;
     c.nbt = p.nblocks;
+    c.tps = 1;
+    c.b_sub = 0;
     c.pre = p.wexp ? 1 : 0;
     // 64-byte k-blocks when a 128-byte row would be at most half used by the (last) channel chunk
     c.bk = (c.pre && (p.Cin % 128 != 0) && (p.Cin % 128 <= 64)) ? 64 : 128;
@@ -819,6 +873,17 @@ bool plan(const Problem& p, TensorCfg& c)
             const int64_t left = kSmemLimit - (1024 + 64 * kMaxRing) - (int64_t)c.nkb * c.a_bytes -
                                  (int64_t)c.epi_warps * kWarpStage;
             c.nB = (int)std::min<int64_t>(kMaxRing, left / c.b_bytes);
+        }
+        c.tps = 1;
+        c.b_sub = c.b_bytes;
+        if (c.ares && c.bk == 64 && c.cpt == 1 && p.kw == 3) {
+            c.tps = 3;
+            c.b_sub = (c.n_mma * c.bk + 1023) / 1024 * 1024;
+            c.b_bytes = c.tps * c.b_sub;
+            const int64_t left = kSmemLimit - (1024 + 64 * kMaxRing) - (int64_t)c.nkb * c.a_bytes -
+                                 (int64_t)c.epi_warps * kWarpStage;
+            c.nB = (int)std::min<int64_t>(kMaxRing, left / c.b_bytes);
+            if (c.nB < 2) { c.tps = 1; c.b_bytes = kTileN * c.bk; c.b_sub = c.b_bytes; c.nB = (int)std::min<int64_t>(kMaxRing, left / c.b_bytes); }
         }
         // Two row blocks per tile pay when K is long (the two accumulators' epilogue is only half
         // hidden behind the next tile's MMAs) and when the halved tile count does not cost more in
