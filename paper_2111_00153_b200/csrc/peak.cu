@@ -43,21 +43,26 @@ __global__ void __launch_bounds__(kPeakThreads, 1) mma_peak_kernel(int is_bf16, 
             return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)64 << 32) | ((uint64_t)1 << 46) |
                    ((uint64_t)2 << 61);
         };
-        const uint64_t ad = desc(sA), bd = desc(sB);
+        // The issuing thread must not be the limiter: the four descriptor pairs of a k-block are
+        // formed once, and the loop over iterations holds nothing but the four instructions.
+        uint64_t ad[4], bd[4];
+        for (int ks = 0; ks < 4; ++ks) { ad[ks] = desc(sA) + 2 * ks; bd[ks] = desc(sB) + 2 * ks; }
         uint32_t phase = 0;
         bool ok = true;
         for (int it = 0; it < iters && ok; ++it) {
             // one "k-block": 4 instructions walking the 128-byte swizzle atom, like the layer kernel
+            if (is_bf16) {
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                if (is_bf16)
+                for (int ks = 0; ks < 4; ++ks)
                     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                                 ::"r"(tmem), "l"(ad + 2 * ks), "l"(bd + 2 * ks), "r"(idesc), "r"(it | ks) : "memory");
-                else
+                                 ::"r"(tmem), "l"(ad[ks]), "l"(bd[ks]), "r"(idesc), "r"(it | ks) : "memory");
+            } else {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
                     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                                  "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-                                 ::"r"(tmem), "l"(ad + 2 * ks), "l"(bd + 2 * ks), "r"(idesc), "r"(it | ks) : "memory");
+                                 ::"r"(tmem), "l"(ad[ks]), "l"(bd[ks]), "r"(idesc), "r"(it | ks) : "memory");
             }
             if ((it & 7) == 7 || it == iters - 1) {
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

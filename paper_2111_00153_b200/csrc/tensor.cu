@@ -498,7 +498,10 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        // The whole warp walks the loops in step (so that ring positions and descriptors are
+        // warp-uniform values); lane 0 alone issues the MMAs and commits.
+        const bool issuer = (lane == 0);
+        {
             uint32_t sa = 0, phA = 0, sb = 0, phB = 0, it = 0;
             const uint64_t desc_a0 = smem_desc_kmajor(sA, cfg.bk), desc_b0 = smem_desc_kmajor(sB, cfg.bk);
             const uint32_t desc_lo0_a = (uint32_t)desc_a0, desc_lo0_b = (uint32_t)desc_b0, desc_hi = (uint32_t)(desc_a0 >> 32);
@@ -513,18 +516,60 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 bool ok = true;
                 int cc = 0;
                 if (cfg.tps > 1) {
-                    // resident weights, several k-blocks per activation stage (never with two row blocks)
-                    for (int kb = 0; kb < cfg.nkb; kb += cfg.tps) {
+                    // resident weights, three 64-byte k-blocks per activation stage (never with two row blocks)
+                    const uint32_t a_step = (uint32_t)cfg.a_bytes >> 4, b_step = (uint32_t)cfg.b_bytes >> 4,
+                                   t_step = (uint32_t)cfg.b_sub >> 4;
+                    uint32_t a_lo = desc_lo0_a, b_lo = desc_lo0_b + sb * b_step;
+                    const bool two = (cfg.last_ksteps == 2);
+                    for (int kb = 0; kb < cfg.nkb; kb += 3) {
                         if (!mbar_wait(bar_fullB + 8 * sb, phB, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        for (int t = 0; t < cfg.tps; ++t) {
-                            const uint64_t ad = smem_desc_kmajor(sA + (uint32_t)(kb + t) * cfg.a_bytes, cfg.bk),
-                                           bd = smem_desc_kmajor(sB + sb * cfg.b_bytes + t * cfg.b_sub, cfg.bk);
-                            for (int ks = 0; ks < cfg.last_ksteps; ++ks)
-                                mma_i8(d_tmem, ad + 2 * ks, bd + 2 * ks, cfg.idesc, (kb | t | ks) ? 1u : 0u);
+                        if (issuer) {
+                            mma_i8_halves(d_tmem, a_lo, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
+                            if (two) mma_i8_halves(d_tmem, a_lo + 2, b_lo + 2, desc_hi, cfg.idesc, 1u);
+                            mma_i8_halves(d_tmem, a_lo + a_step, b_lo + t_step, desc_hi, cfg.idesc, 1u);
+                            if (two) mma_i8_halves(d_tmem, a_lo + a_step + 2, b_lo + t_step + 2, desc_hi, cfg.idesc, 1u);
+                            mma_i8_halves(d_tmem, a_lo + 2 * a_step, b_lo + 2 * t_step, desc_hi, cfg.idesc, 1u);
+                            if (two) mma_i8_halves(d_tmem, a_lo + 2 * a_step + 2, b_lo + 2 * t_step + 2, desc_hi, cfg.idesc, 1u);
+                            mma_commit(bar_emptyB + 8 * sb);
                         }
-                        mma_commit(bar_emptyB + 8 * sb);
-                        if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; }
+                        a_lo += 3 * a_step;
+                        b_lo += b_step;
+                        if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; b_lo = desc_lo0_b; }
+                    }
+                } else if (!cfg.ares && cfg.bk == 128 && cfg.last_ksteps == 4) {
+                    // The common deep-K form, kept as short as it gets: every k-block is four MMAs (eight
+                    // with two row blocks) on a full 128-byte stage of each ring.
+                    const uint32_t a_step = (uint32_t)cfg.a_bytes >> 4, b_step = (uint32_t)cfg.b_bytes >> 4;
+                    uint32_t a_lo = desc_lo0_a + sa * a_step, b_lo = desc_lo0_b + sb * b_step;
+                    if (kM2) {
+                        if (!mbar_wait(bar_tempty + 8, tpar, abort_flag)) break;
+                        tc_fence_after();
+                    }
+                    for (int kb = 0; kb < cfg.nkb; ++kb) {
+                        if (!mbar_wait(bar_fullB + 8 * sb, phB, abort_flag) || !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t acc = kb ? 1u : 0u;
+                        if (issuer) mma_i8_halves(d_tmem, a_lo, b_lo, desc_hi, cfg.idesc, acc);
+                        if (issuer) mma_i8_halves(d_tmem, a_lo + 2, b_lo + 2, desc_hi, cfg.idesc, 1u);
+                        if (issuer) mma_i8_halves(d_tmem, a_lo + 4, b_lo + 4, desc_hi, cfg.idesc, 1u);
+                        if (issuer) mma_i8_halves(d_tmem, a_lo + 6, b_lo + 6, desc_hi, cfg.idesc, 1u);
+                        if (kM2) {
+                            const uint32_t a1 = a_lo + (kABytes >> 4);
+                            if (issuer) mma_i8_halves(d_tmem + kTileN, a1, b_lo, desc_hi, cfg.idesc, acc);
+                            if (issuer) mma_i8_halves(d_tmem + kTileN, a1 + 2, b_lo + 2, desc_hi, cfg.idesc, 1u);
+                            if (issuer) mma_i8_halves(d_tmem + kTileN, a1 + 4, b_lo + 4, desc_hi, cfg.idesc, 1u);
+                            if (issuer) mma_i8_halves(d_tmem + kTileN, a1 + 6, b_lo + 6, desc_hi, cfg.idesc, 1u);
+                        }
+                        if (issuer) mma_commit(bar_emptyA + 8 * sa);
+                        if (issuer) mma_commit(bar_emptyB + 8 * sb);
+                        a_lo += a_step;
+                        b_lo += b_step;
+                        if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; a_lo = desc_lo0_a; }
+                        if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; b_lo = desc_lo0_b; }
                     }
                 } else {
                     const bool uniform = (cfg.last_ksteps == (cfg.bk >> 5));      // every k-block has the same depth
@@ -536,9 +581,9 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                             (!cfg.ares && !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag))) { ok = false; break; }
                         tc_fence_after();
                         const int ksteps = (uniform || cc != cfg.cpt - 1) ? (cfg.bk >> 5) : cfg.last_ksteps;
-                        mma_i8_halves(d_tmem, a_lo, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
+                        if (issuer) mma_i8_halves(d_tmem, a_lo, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
                         for (int ks = 1; ks < ksteps; ++ks)
-                            mma_i8_halves(d_tmem, a_lo + 2 * ks, b_lo + 2 * ks, desc_hi, cfg.idesc, 1u);
+                            if (issuer) mma_i8_halves(d_tmem, a_lo + 2 * ks, b_lo + 2 * ks, desc_hi, cfg.idesc, 1u);
                         if (kM2) {
                             // second row block: rows 128..255 of the weight stage, second accumulator
                             if (kb == 0) {
@@ -546,12 +591,12 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                                 tc_fence_after();
                             }
                             const uint32_t a1 = a_lo + (kABytes >> 4);
-                            mma_i8_halves(d_tmem + kTileN, a1, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
+                            if (issuer) mma_i8_halves(d_tmem + kTileN, a1, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
                             for (int ks = 1; ks < ksteps; ++ks)
-                                mma_i8_halves(d_tmem + kTileN, a1 + 2 * ks, b_lo + 2 * ks, desc_hi, cfg.idesc, 1u);
+                                if (issuer) mma_i8_halves(d_tmem + kTileN, a1 + 2 * ks, b_lo + 2 * ks, desc_hi, cfg.idesc, 1u);
                         }
-                        if (!cfg.ares) mma_commit(bar_emptyA + 8 * sa);
-                        mma_commit(bar_emptyB + 8 * sb);
+                        if (!cfg.ares && issuer) mma_commit(bar_emptyA + 8 * sa);
+                        if (issuer) mma_commit(bar_emptyB + 8 * sb);
                         a_lo += a_step;
                         b_lo += b_step;
                         if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; if (!cfg.ares) a_lo = desc_lo0_a; }
@@ -560,8 +605,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                     }
                 }
                 if (!ok) break;
-                mma_commit(bar_tfull + 8 * ab);
-                if (kM2) mma_commit(bar_tfull + 8);
+                if (issuer) mma_commit(bar_tfull + 8 * ab);
+                if (kM2 && issuer) mma_commit(bar_tfull + 8);
             }
         }
     } else if (!cfg.pre && warp < 2 + kNumExpWarps) {
@@ -876,7 +921,7 @@ bool plan(const Problem& p, TensorCfg& c)
         }
         c.tps = 1;
         c.b_sub = c.b_bytes;
-        if (c.ares && c.bk == 64 && c.cpt == 1 && p.kw == 3) {
+        if (c.ares && c.bk == 64 && c.cpt == 1 && p.kw == 3 && c.last_ksteps <= 2) {
             c.tps = 3;
             c.b_sub = (c.n_mma * c.bk + 1023) / 1024 * 1024;
             c.b_bytes = c.tps * c.b_sub;
