@@ -54,6 +54,8 @@ struct Problem {
 // kernels (each returns the CUDA launch error, cudaSuccess if fine)
 cudaError_t launch_pack(const float* dW, int conv_oihw, const rmsmp_layer& L, int pot_mode,
                         uint8_t* blob, cudaStream_t st);
+// copies `bytes` from mapped pinned host memory (device view, 16-byte aligned) to device memory
+cudaError_t launch_fetch_mapped(void* d_dst, const void* mapped_src, size_t bytes, cudaStream_t st);
 cudaError_t launch_unpack(const rmsmp_layer& L, const uint8_t* blob, int8_t* values,
                           int32_t* perm, float* wstep, cudaStream_t st);
 cudaError_t launch_expand(const rmsmp_layer& L, const uint8_t* blob, int8_t* wexp, cudaStream_t st);

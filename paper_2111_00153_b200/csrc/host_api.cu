@@ -46,15 +46,20 @@ rmsmp_status check_arch()
 }
 
 // Pinned host staging for the metadata upload of rmsmp_quantize_pack.  A copy from pageable memory
-// makes the host wait for the stream; from pinned memory it is asynchronous.  One small ring of
+// makes the host wait for the stream; from pinned memory it is asynchronous.  The slot is mapped
+// into the device's address space and a small kernel fetches it: between two kernels of a stream a
+// copy-engine transfer of a few KB costs several microseconds more than a kernel does.  One small ring of
 // slots per device, created on first use (host memory only; no device memory is ever allocated);
 // an event per slot tells when its last copy has left.  If pinned memory cannot be had, or the
 // metadata is larger than a slot, the pageable path is used.
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
 constexpr size_t kStageSlotBytes = 64 * 1024;
 constexpr int kStageSlots = 32;
 struct StageRing {
     bool tried = false;
     uint8_t* base = nullptr;
+    uint8_t* dev_base = nullptr;      // the same memory as the device sees it
     cudaEvent_t ev[kStageSlots];
     bool used[kStageSlots];
     int next = 0;
@@ -73,7 +78,7 @@ bool staged_upload(void* d_dst, const void* h_src, size_t bytes, cudaStream_t st
     if (!r.tried) {
         r.tried = true;
         void* ptr = nullptr;
-        if (cudaHostAlloc(&ptr, kStageSlotBytes * kStageSlots, cudaHostAllocDefault) != cudaSuccess) {
+        if (cudaHostAlloc(&ptr, kStageSlotBytes * kStageSlots, cudaHostAllocMapped) != cudaSuccess) {
             cudaGetLastError();
         } else {
             bool ok = true;
@@ -81,7 +86,9 @@ bool staged_upload(void* d_dst, const void* h_src, size_t bytes, cudaStream_t st
                 r.used[i] = false;
                 if (cudaEventCreateWithFlags(&r.ev[i], cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); ok = false; break; }
             }
-            if (ok) r.base = static_cast<uint8_t*>(ptr); else cudaFreeHost(ptr);
+            void* dptr = nullptr;
+            if (ok && cudaHostGetDevicePointer(&dptr, ptr, 0) != cudaSuccess) { cudaGetLastError(); dptr = nullptr; }
+            if (ok) { r.base = static_cast<uint8_t*>(ptr); r.dev_base = static_cast<uint8_t*>(dptr); } else cudaFreeHost(ptr);
         }
     }
     if (!r.base) return false;
@@ -90,13 +97,16 @@ bool staged_upload(void* d_dst, const void* h_src, size_t bytes, cudaStream_t st
     if (r.used[slot] && cudaEventSynchronize(r.ev[slot]) != cudaSuccess) { cudaGetLastError(); return false; }
     uint8_t* h = r.base + (size_t)slot * kStageSlotBytes;
     std::memcpy(h, h_src, bytes);
-    if (cudaMemcpyAsync(d_dst, h, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); return false; }
+    const bool by_kernel = r.dev_base && aligned16(d_dst) &&
+                           launch_fetch_mapped(d_dst, r.dev_base + (size_t)slot * kStageSlotBytes, bytes, st) == cudaSuccess;
+    if (!by_kernel) {
+        cudaGetLastError();
+        if (cudaMemcpyAsync(d_dst, h, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); return false; }
+    }
     if (cudaEventRecord(r.ev[slot], st) != cudaSuccess) { cudaGetLastError(); return false; }
     r.used[slot] = true;
     return true;
 }
-
-inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 void fill_problem(Problem& p, const rmsmp_layer* L, const void* d_packed)
 {

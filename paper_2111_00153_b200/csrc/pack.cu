@@ -90,9 +90,19 @@ __global__ void __launch_bounds__(256) pack_kernel(PackArgs a)
             s_code[kp - seg0] = (uint8_t)code;
         };
         if (vec4) {
-            for (int idx = k_lo + threadIdx.x * 4; idx < k_hi; idx += blockDim.x * 4) {
-                float4 w = *reinterpret_cast<const float4*>(wrow + idx);
-                put(idx, w.x); put(idx + 1, w.y); put(idx + 2, w.z); put(idx + 3, w.w);
+            // four 128-bit loads in flight per thread before any code is formed: a block walks one
+            // row, so its time is the number of dependent load rounds
+            const int stride = blockDim.x * 4;
+            for (int idx0 = k_lo + threadIdx.x * 4; idx0 < k_hi; idx0 += 4 * stride) {
+                float4 w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (idx0 + u * stride < k_hi) w[u] = __ldg(reinterpret_cast<const float4*>(wrow + idx0 + u * stride));
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int idx = idx0 + u * stride;
+                    if (idx < k_hi) { put(idx, w[u].x); put(idx + 1, w[u].y); put(idx + 2, w[u].z); put(idx + 3, w[u].w); }
+                }
             }
         } else {
             for (int idx = k_lo + threadIdx.x; idx < k_hi; idx += blockDim.x) put(idx, wrow[idx]);
@@ -144,10 +154,35 @@ cudaError_t launch_pack(const float* dW, int conv_oihw, const rmsmp_layer& L, in
     a.pot_mode = pot_mode;
     a.seg = a.conv ? L.Kp : (L.Kp < 32768 ? L.Kp : 32768);
     size_t smem = (size_t)a.seg;
-    cudaError_t e = cudaFuncSetAttribute(pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(smem > 48 * 1024 ? smem : 48 * 1024));
-    if (e != cudaSuccess) return e;
+    if (smem > 48 * 1024) {            // rows longer than the default dynamic shared memory limit
+        cudaError_t e = cudaFuncSetAttribute(pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
     pack_kernel<<<L.M, 256, smem, st>>>(a);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ metadata fetch
+// The few KB of per-row metadata come from mapped pinned host memory: 128-bit reads across the
+// host link, 128-bit writes to the packed buffer.
+
+__global__ void __launch_bounds__(256) fetch_mapped_kernel(uint8_t* __restrict__ dst, const uint8_t* __restrict__ src,
+                                                           size_t bytes)
+{
+    const size_t n16 = bytes / 16;
+    const size_t tid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, nthr = (size_t)gridDim.x * blockDim.x;
+    // host memory: loads that bypass the caches, so that a reused slot is never read stale
+    for (size_t i = tid; i < n16; i += nthr)
+        reinterpret_cast<uint4*>(dst)[i] = __ldcv(reinterpret_cast<const uint4*>(src) + i);
+    for (size_t i = n16 * 16 + tid; i < bytes; i += nthr) dst[i] = __ldcv(src + i);
+}
+
+cudaError_t launch_fetch_mapped(void* d_dst, const void* mapped_src, size_t bytes, cudaStream_t st)
+{
+    size_t blocks = (bytes / 16 + 255) / 256;
+    if (blocks > 64) blocks = 64;
+    if (blocks == 0) blocks = 1;
+    fetch_mapped_kernel<<<(unsigned)blocks, 256, 0, st>>>(static_cast<uint8_t*>(d_dst), static_cast<const uint8_t*>(mapped_src), bytes);
     return cudaGetLastError();
 }
 
