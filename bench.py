@@ -480,6 +480,28 @@ def run_suite(args):
     for ratio in synth.RATIO_SWEEP:
         bench_shape("config5", "bert-large ffn1 4096x1024 N=8 ratio %d:%d:%d" % ratio, 4096, 1024, 1, 1, 0, 8, 1,
                     ratio=ratio, pool=24, only=("simt_dp4a", "shift_add"), iters=48)
+    # config 5 as the natural cold stream: the whole BERT-large stack (24 x six linears, ~158 MB of
+    # packed weights, larger than L2) in ONE grouped launch; the table upload is part of the call.
+    for N in (1, 8):
+        keep, items, wbytes, ops, alg = [], [], 0, 0, 0
+        for l in range(24):
+            for (M, K) in ((1024, 1024),) * 4 + ((4096, 1024), (1024, 4096)):
+                lay, pk, _ = prep(M, K, 1, RATIO, 1000 + 7 * l + M // 1000 + K // 500, False)
+                act = torch.randint(0, 16, (N, K), dtype=torch.int8, device="cuda")
+                yy = torch.empty((N, M), dtype=torch.float32, device="cuda")
+                keep.append((lay, pk, act, yy))
+                items.append((lay, pk, act, N, K, 0.1, yy, M, None))
+                ops += 2 * M * K * N
+                alg += (lay.nP + lay.nF4) * K // 2 + lay.n8 * K + 8 * M + N * K + 4 * N * M
+        arr = R.make_gemm_items(items)
+        table = torch.empty(R.rmsmp_grouped_table_bytes(len(items)), dtype=torch.uint8, device="cuda")
+        us = timed(lambda i: R.rmsmp_gemm_grouped(arr, R.OUT_NM, table), 8)
+        rec = {"suite": "config5", "shape": "bert-large stack, 144 linears, N=%d, one grouped launch" % N, "N": N,
+               "ratio": list(RATIO), "variant": "grouped_dp4a", "us": us, "tops": ops / us / 1e6, "gbs": alg / us / 1e3,
+               "frac_int8_peak": ops / us / 1e6 / i8_peak, "frac_hbm": alg / us / 1e3 / peaks["hbm_gbs"], "weights": "cold stream"}
+        rows.append(rec)
+        print(json.dumps(rec))
+        del keep, items, arr, table
     print("\n| config | shape | variant | us | TOPS | GB/s | of INT8 peak | of HBM |")
     print("|---|---|---|---|---|---|---|---|")
     for r in rows:
