@@ -196,18 +196,40 @@ def run_ours(args):
             R.rmsmp_conv_implicit_variant(h["lay"], d["packed"], d["codes"], batch, L.H, L.H, L.stride, L.pad, st,
                                           d["y"], R.OUT_NM, None, R.VARIANT_TENSOR, stream=stream)
 
+    # Two streams: the weight path of a layer (quantize_pack + expand_weights: three small,
+    # latency-bound launches) does not depend on its activations, so it runs on a side stream and
+    # overlaps the activation quantizer / the previous layer's tail.  The convolution waits for
+    # both; the next step's pack of a layer waits for this step's convolution of it (same buffers).
+    side = torch.cuda.Stream() if args.streams == 2 else None
+    ready = [torch.cuda.Event() for _ in layers]
+    done = [torch.cuda.Event() for _ in layers]
+    first_use = [True]
+
     def step(ev=None):
         for i, (h, d) in enumerate(zip(H, D)):
+            ws_stream = side if side is not None else stream
+            if side is not None:
+                if first_use[0]:
+                    side.wait_stream(stream)
+                else:
+                    side.wait_event(done[i])
             R.rmsmp_quantize_pack(d["W"], R.W_CONV_OIHW, h["lay"], h["scheme"], h["bits"], h["alpha"],
-                                  R.POT_NEAREST, d["packed"], stream=stream)
+                                  R.POT_NEAREST, d["packed"], stream=ws_stream)
             if use_ws:
-                R.rmsmp_expand_weights(h["lay"], d["packed"], d["ws"], stream=stream)
+                R.rmsmp_expand_weights(h["lay"], d["packed"], d["ws"], stream=ws_stream)
+            if side is not None:
+                ready[i].record(side)
             st = R.rmsmp_quantize_act(d["x"], d["x"].numel(), synth.ALPHA_ACT, R.ACT_U4, d["codes"], stream=stream)
+            if side is not None:
+                stream.wait_event(ready[i])
             if ev is not None:
                 ev[i][0].record(stream)
             conv(h, d, st)
             if ev is not None:
                 ev[i][1].record(stream)
+            if side is not None:
+                done[i].record(stream)
+        first_use[0] = False
 
     def barrier():
         if world > 1:
@@ -292,7 +314,8 @@ def run_ours(args):
         "data": "synthetic",
         "config": {"workload": WORKLOAD if LAYER_FILTER is None else "subset:" + ",".join(sorted(LAYER_FILTER)), "batch_per_gpu": batch, "layers": len(layers),
                    "ops_per_step_per_gpu": ops_step, "l2": "inputs larger than L2 (every layer reads 13-205 MB and writes 6-205 MB)",
-                   "step": "per layer: quantize_pack%s + quantize_act + conv_implicit (tensor cores, %s)" % ((" + expand_weights", "weights expanded once into scratch") if use_ws else ("", "weights expanded in shared memory per tile"))},
+                   "step": "per layer: quantize_pack%s + quantize_act + conv_implicit (tensor cores, %s)" % ((" + expand_weights", "weights expanded once into scratch") if use_ws else ("", "weights expanded in shared memory per tile")),
+                   "streams": args.streams},
         "clocks": clocks,
         "e2e": ({"value": whole_job_tops(ops_step, world, e2e_ms_step), "unit": UNIT, "ms_per_step": e2e_ms_step,
                  "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h} if e2e_steps else None),
@@ -523,6 +546,9 @@ def main():
     ap.add_argument("--variant", default="workspace", choices=["workspace", "smem"],
                     help="tensor-core path: expand the weight codes once into scratch memory (default) "
                          "or in shared memory per tile")
+    ap.add_argument("--streams", type=int, default=2, choices=[1, 2],
+                    help="2: each layer's weight path (pack, expand) runs on a side stream and overlaps the "
+                         "activation path; 1: everything on one stream")
     ap.add_argument("--suite", action="store_true",
                     help="side-by-side timing of the kernel variants on all five configurations (not the headline)")
     ap.add_argument("--layers", default=None,
