@@ -259,6 +259,33 @@ rmsmp_status rmsmp_conv_implicit_workspace(const rmsmp_layer* layer, const void*
                                            int32_t* d_acc, void* stream);
 
 /*
+ * Layer chaining without the fp32 round trip.  The paper runs the quantized model layer by layer
+ * with 4-bit activations between layers (Section 3.1, Algorithm 1's forward pass); these calls
+ * fuse the NEXT layer's activation quantizer into the epilogue: instead of
+ * y[n][m] = float(acc) * (wstep_m * act_step) they write the 4-bit code of that same y,
+ *     d_next_codes[n * ld_codes + m] = code(y[n][m]; next_alpha, next_kind),
+ * with exactly the arithmetic of rmsmp_quantize_act (RMSMP_ACT_U4 clips at 0, which is the ReLU;
+ * RMSMP_ACT_S4 keeps the sign), so the result equals rmsmp_*_workspace followed by
+ * rmsmp_quantize_act byte for byte while writing 1 byte per output instead of 4 and saving the
+ * quantizer's pass.  [N][M] order only (conv: [B][Ho][Wo][M], ld_codes = M): that is the next
+ * layer's input layout.  d_next_codes: device, N * ld_codes bytes; bulk stores are used when it is
+ * 16-byte aligned and ld_codes is a multiple of 16.  *h_next_step (host, may be NULL) receives
+ * next_alpha/15 or next_alpha/7.  Errors: as rmsmp_*_workspace, plus SCALE for a bad next_alpha;
+ * VARIANT when the tensor kernel cannot run the problem.
+ */
+rmsmp_status rmsmp_gemm_workspace_requant(const rmsmp_layer* layer, const void* d_packed,
+                                          const void* d_workspace, const int8_t* d_act, int64_t N,
+                                          int64_t ld_act, float act_step, float next_alpha,
+                                          rmsmp_act_kind next_kind, int8_t* d_next_codes,
+                                          int64_t ld_codes, float* h_next_step, void* stream);
+rmsmp_status rmsmp_conv_implicit_workspace_requant(const rmsmp_layer* layer, const void* d_packed,
+                                                   const void* d_workspace, const int8_t* d_act,
+                                                   int B, int H, int W, int stride, int pad,
+                                                   float act_step, float next_alpha,
+                                                   rmsmp_act_kind next_kind, int8_t* d_next_codes,
+                                                   float* h_next_step, void* stream);
+
+/*
  * Linear layer for callers that cannot allocate device memory (the paper has no counterpart:
  * this is a deployment convenience of the library).  Same computation and same results as
  * rmsmp_expand_weights followed by rmsmp_gemm_workspace, but the scratch for the expanded

@@ -31,7 +31,7 @@ EXPORTS = (
     "rmsmp_conv_implicit", "rmsmp_conv_implicit_variant", "rmsmp_last_device_status",
     "rmsmp_measure_mma_peak", "rmsmp_workspace_bytes", "rmsmp_expand_weights", "rmsmp_gemm_workspace",
     "rmsmp_conv_implicit_workspace", "rmsmp_gemm_builtin_scratch", "rmsmp_grouped_table_bytes",
-    "rmsmp_gemm_grouped",
+    "rmsmp_gemm_grouped", "rmsmp_gemm_workspace_requant", "rmsmp_conv_implicit_workspace_requant",
 )
 
 
@@ -108,6 +108,10 @@ def lib() -> C.CDLL:
         L.rmsmp_gemm_builtin_scratch.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
         L.rmsmp_conv_implicit_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
                                                     f32, vp, i32, vp, vp]
+        L.rmsmp_gemm_workspace_requant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i64, i64, f32, f32, i32, vp, i64,
+                                                   C.POINTER(C.c_float), vp]
+        L.rmsmp_conv_implicit_workspace_requant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
+                                                            f32, f32, i32, vp, C.POINTER(C.c_float), vp]
         L.rmsmp_measure_mma_peak.argtypes = [i32, i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
         _lib = L
     return _lib
@@ -222,6 +226,27 @@ def rmsmp_conv_implicit_variant(layer, d_packed, d_act, B: int, H: int, W: int, 
                                              stride, pad, act_step, _dp(d_out), out_layout,
                                              _dp(d_acc), variant, _stream(stream)),
            "rmsmp_conv_implicit_variant")
+
+
+def rmsmp_gemm_workspace_requant(layer, d_packed, d_workspace, d_act, N: int, ld_act: int, act_step: float,
+                                 next_alpha: float, next_kind: int, d_next_codes, ld_codes: int, stream=None) -> float:
+    """Linear layer whose epilogue writes the next layer's 4-bit activation codes; returns their step."""
+    step = C.c_float(0.0)
+    _check(lib().rmsmp_gemm_workspace_requant(C.byref(layer), _dp(d_packed), _dp(d_workspace), _dp(d_act), N, ld_act,
+                                              act_step, next_alpha, next_kind, _dp(d_next_codes), ld_codes,
+                                              C.byref(step), _stream(stream)), "rmsmp_gemm_workspace_requant")
+    return step.value
+
+
+def rmsmp_conv_implicit_workspace_requant(layer, d_packed, d_workspace, d_act, B: int, H: int, W: int, stride: int,
+                                          pad: int, act_step: float, next_alpha: float, next_kind: int,
+                                          d_next_codes, stream=None) -> float:
+    step = C.c_float(0.0)
+    _check(lib().rmsmp_conv_implicit_workspace_requant(C.byref(layer), _dp(d_packed), _dp(d_workspace), _dp(d_act),
+                                                       B, H, W, stride, pad, act_step, next_alpha, next_kind,
+                                                       _dp(d_next_codes), C.byref(step), _stream(stream)),
+           "rmsmp_conv_implicit_workspace_requant")
+    return step.value
 
 
 def rmsmp_workspace_bytes(layer) -> int:

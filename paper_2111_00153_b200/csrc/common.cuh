@@ -49,6 +49,12 @@ struct Problem {
     int32_t* acc;             // may be null
     int64_t ld_out;
     int out_mn;               // 0: y[n*ld+m], 1: y[m*ld+n]
+    // re-quantizing epilogue (tensor path, workspace mode): when rq_codes is set the kernel writes
+    // the NEXT layer's 4-bit activation codes of y, codes[n*ld_codes+m], instead of y itself
+    int8_t* rq_codes;
+    float rq_alpha;
+    int rq_kind;
+    int64_t ld_codes;
 };
 
 // kernels (each returns the CUDA launch error, cudaSuccess if fine)

@@ -124,6 +124,7 @@ void fill_problem(Problem& p, const rmsmp_layer* L, const void* d_packed)
     p.nP = L->nP; p.nF4 = L->nF4; p.n8 = L->n8; p.nblocks = L->nblocks;
     p.raw_stage_bytes = L->raw_stage_bytes;
     p.wexp = nullptr;
+    p.rq_codes = nullptr; p.rq_alpha = 1.0f; p.rq_kind = 0; p.ld_codes = 0;
 }
 
 rmsmp_status dispatch(Problem& p, rmsmp_variant variant, cudaStream_t st)
@@ -344,19 +345,37 @@ rmsmp_status rmsmp_quantize_act(const float* d_X, size_t count, float alpha_a, r
     return RMSMP_OK;
 }
 
+// Re-quantizing epilogue request (rmsmp_*_workspace_requant): the next layer's clip value, kind and code buffer.
+struct Requant {
+    float alpha;
+    rmsmp_act_kind kind;
+    int8_t* codes;
+    int64_t ld;
+};
+
+static rmsmp_status requant_check(const Requant* rq, float* h_next_step)
+{
+    if (!rq->codes) return RMSMP_ERR_NULL;
+    if (rq->kind != RMSMP_ACT_U4 && rq->kind != RMSMP_ACT_S4) return RMSMP_ERR_SCHEME;
+    if (!(rq->alpha > 0.0f) || !std::isfinite(rq->alpha)) return RMSMP_ERR_SCALE;
+    if (h_next_step) *h_next_step = rq->alpha / (rq->kind == RMSMP_ACT_U4 ? 15.0f : 7.0f);
+    return RMSMP_OK;
+}
+
 static rmsmp_status gemm_impl(const rmsmp_layer* L, const void* d_packed, const void* d_ws, bool use_ws,
                               const int8_t* d_act, int64_t N, int64_t ld_act, float act_step, float* d_out,
                               int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
-                              rmsmp_variant variant, void* stream)
+                              rmsmp_variant variant, void* stream, const Requant* rq = nullptr)
 {
-    if (!L || !d_packed || !d_act || !d_out || (use_ws && !d_ws)) return RMSMP_ERR_NULL;
+    if (!L || !d_packed || !d_act || (!d_out && !rq) || (use_ws && !d_ws)) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     if (L->kh != 1 || L->kw != 1) return RMSMP_ERR_SHAPE;
     if (N < 1 || N > (int64_t)1 << 31 || ld_act < L->Cin) return RMSMP_ERR_SHAPE;
     if (out_layout != RMSMP_OUT_NM && out_layout != RMSMP_OUT_MN) return RMSMP_ERR_SHAPE;
-    if (ld_out < (out_layout == RMSMP_OUT_NM ? (int64_t)L->M : N)) return RMSMP_ERR_SHAPE;
+    if (!rq && ld_out < (out_layout == RMSMP_OUT_NM ? (int64_t)L->M : N)) return RMSMP_ERR_SHAPE;
+    if (rq && rq->ld < L->M) return RMSMP_ERR_SHAPE;
     if (!std::isfinite(act_step)) return RMSMP_ERR_SCALE;
-    if (!aligned16(d_act) || !aligned16(d_out) || (d_acc && !aligned16(d_acc)) || (ld_act & 15) ||
+    if (!aligned16(d_act) || (!rq && !aligned16(d_out)) || (d_acc && !aligned16(d_acc)) || (ld_act & 15) ||
         (reinterpret_cast<uintptr_t>(d_packed) & 255))
         return RMSMP_ERR_ALIGN;
     rmsmp_status a = check_arch();
@@ -368,6 +387,7 @@ static rmsmp_status gemm_impl(const rmsmp_layer* L, const void* d_packed, const 
     p.pix_pitch = ld_act; p.N = N;
     p.act_step = act_step; p.out = d_out; p.acc = d_acc; p.ld_out = ld_out;
     p.out_mn = (out_layout == RMSMP_OUT_MN);
+    if (rq) { p.rq_codes = rq->codes; p.rq_alpha = rq->alpha; p.rq_kind = rq->kind; p.ld_codes = rq->ld; }
     if (use_ws) {
         if (!aligned16(d_ws)) return RMSMP_ERR_ALIGN;
         p.wexp = static_cast<const int8_t*>(d_ws);
@@ -460,9 +480,9 @@ rmsmp_status rmsmp_gemm(const rmsmp_layer* L, const void* d_packed, const int8_t
 static rmsmp_status conv_impl(const rmsmp_layer* L, const void* d_packed, const void* d_ws, bool use_ws,
                               const int8_t* d_act, int B, int H, int W, int stride, int pad, float act_step,
                               float* d_out, rmsmp_out_layout out_layout, int32_t* d_acc,
-                              rmsmp_variant variant, void* stream)
+                              rmsmp_variant variant, void* stream, const Requant* rq = nullptr)
 {
-    if (!L || !d_packed || !d_act || !d_out || (use_ws && !d_ws)) return RMSMP_ERR_NULL;
+    if (!L || !d_packed || !d_act || (!d_out && !rq) || (use_ws && !d_ws)) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     if (B < 1 || H < 1 || W < 1 || stride < 1 || stride > 8 || pad < 0 || pad > 16) return RMSMP_ERR_SHAPE;
     if (H + 2 * pad < L->kh || W + 2 * pad < L->kw) return RMSMP_ERR_SHAPE;
@@ -471,7 +491,7 @@ static rmsmp_status conv_impl(const rmsmp_layer* L, const void* d_packed, const 
     const int Ho = (H + 2 * pad - L->kh) / stride + 1, Wo = (W + 2 * pad - L->kw) / stride + 1;
     const int64_t N = (int64_t)B * Ho * Wo;
     if (N > (int64_t)1 << 31 || (int64_t)B * H * W > (int64_t)1 << 31) return RMSMP_ERR_SHAPE;
-    if (!aligned16(d_act) || !aligned16(d_out) || (d_acc && !aligned16(d_acc)) ||
+    if (!aligned16(d_act) || (!rq && !aligned16(d_out)) || (d_acc && !aligned16(d_acc)) ||
         (reinterpret_cast<uintptr_t>(d_packed) & 255))
         return RMSMP_ERR_ALIGN;
     rmsmp_status a = check_arch();
@@ -484,6 +504,7 @@ static rmsmp_status conv_impl(const rmsmp_layer* L, const void* d_packed, const 
     p.act_step = act_step; p.out = d_out; p.acc = d_acc;
     p.out_mn = (out_layout == RMSMP_OUT_MN);
     p.ld_out = p.out_mn ? N : L->M;
+    if (rq) { p.rq_codes = rq->codes; p.rq_alpha = rq->alpha; p.rq_kind = rq->kind; p.ld_codes = L->M; }
     if (use_ws) {
         if (!aligned16(d_ws)) return RMSMP_ERR_ALIGN;
         p.wexp = static_cast<const int8_t*>(d_ws);
@@ -508,6 +529,31 @@ rmsmp_status rmsmp_conv_implicit_workspace(const rmsmp_layer* L, const void* d_p
 {
     return conv_impl(L, d_packed, d_workspace, true, d_act, B, H, W, stride, pad, act_step, d_out, out_layout,
                      d_acc, RMSMP_VARIANT_TENSOR, stream);
+}
+
+rmsmp_status rmsmp_gemm_workspace_requant(const rmsmp_layer* L, const void* d_packed, const void* d_workspace,
+                                          const int8_t* d_act, int64_t N, int64_t ld_act, float act_step,
+                                          float next_alpha, rmsmp_act_kind next_kind, int8_t* d_next_codes,
+                                          int64_t ld_codes, float* h_next_step, void* stream)
+{
+    const Requant rq = {next_alpha, next_kind, d_next_codes, ld_codes};
+    rmsmp_status s = requant_check(&rq, h_next_step);
+    if (s != RMSMP_OK) return s;
+    return gemm_impl(L, d_packed, d_workspace, true, d_act, N, ld_act, act_step, nullptr, 0, RMSMP_OUT_NM, nullptr,
+                     RMSMP_VARIANT_TENSOR, stream, &rq);
+}
+
+rmsmp_status rmsmp_conv_implicit_workspace_requant(const rmsmp_layer* L, const void* d_packed,
+                                                   const void* d_workspace, const int8_t* d_act, int B, int H,
+                                                   int W, int stride, int pad, float act_step, float next_alpha,
+                                                   rmsmp_act_kind next_kind, int8_t* d_next_codes,
+                                                   float* h_next_step, void* stream)
+{
+    const Requant rq = {next_alpha, next_kind, d_next_codes, 0};
+    rmsmp_status s = requant_check(&rq, h_next_step);
+    if (s != RMSMP_OK) return s;
+    return conv_impl(L, d_packed, d_workspace, true, d_act, B, H, W, stride, pad, act_step, nullptr, RMSMP_OUT_NM,
+                     nullptr, RMSMP_VARIANT_TENSOR, stream, &rq);
 }
 
 rmsmp_status rmsmp_workspace_bytes(const rmsmp_layer* L, size_t* bytes)

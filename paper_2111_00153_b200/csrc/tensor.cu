@@ -28,6 +28,7 @@
 #include <cstring>
 #include "common.cuh"
 #include "decode.cuh"
+#include "actq.cuh"
 
 namespace rmsmp {
 
@@ -87,6 +88,7 @@ struct Maps {
     CUtensorMap q4, q8;                                // packed weight regions
     CUtensorMap wexp;                                  // [M][Kp] int8 weights expanded beforehand (pre mode); 64-row box when dup
     CUtensorMap out_full, out_tail, acc_full, acc_tail;   // bulk stores: 32-row and tail chunks
+    CUtensorMap rq_full, rq_tail;                       // re-quantized codes: 32 pixels x 32 code bytes, and the tail
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -298,7 +300,8 @@ __device__ __forceinline__ void expand_task(uint32_t meta, uint32_t raw_stage, u
 // ------------------------------------------------------------------ the kernel
 
 // kM2: a tile covers two row blocks (TensorCfg::m2), compiled separately so that the common form keeps its registers.
-template <int kM2>
+// kRQ: the epilogue writes the next layer's activation codes instead of fp32 (Problem::rq_codes).
+template <int kM2, int kRQ>
 __global__ void __launch_bounds__(kThreads, 1)
 tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps maps)
 {
@@ -686,6 +689,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         const uint32_t my_stage = sOut + (uint32_t)ew * (cfg.out_bufs * kWarpStage);
         uint32_t it = 0, stg_count = 0;
         bool alive = true;
+        const ActFast rq_fast = act_fast_setup(kRQ ? p.rq_alpha : 1.0f, kRQ ? p.rq_kind : 0);
         for (int64_t tile = first; tile < cfg.ntiles && alive; tile += step, ++it) {
           // a tile is one row block (accumulators alternate between tiles), or two (one accumulator each)
           for (int half = 0; half <= kM2; ++half) {
@@ -722,7 +726,34 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
             // Output one 32-pixel chunk held in registers.
             auto emit = [&](const uint32_t (&v)[32], int c) {
                 const int jmax = min(32, nvalid - c * 32);
-                if (cfg.tma_store) {
+                if (kRQ) {
+                    // y as in the fp32 epilogue, then the activation quantizer's arithmetic on it;
+                    // one code byte per output, 32 pixels x 32 rows = 1 KB per chunk
+                    if (cfg.tma_store) {
+                        const bool tail = cfg.tail_rows && (c == (cfg.npix >> 5));
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float y = __fmul_rn(__int2float_rn((int)v[j] >> shift), scale);
+                            const uint32_t code = act_code_exact(y, p.rq_alpha, p.rq_kind, rq_fast);
+                            asm volatile("st.shared.u8 [%0], %1;" ::"r"(my_stage + j * 32 + lane), "r"(code) : "memory");
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0)
+                            tma_store_2d(tail ? &maps.rq_tail : &maps.rq_full, my_stage, blk * kBlockRows + row0, (int)(n0 + c * 32));
+                    } else if (row_ok) {
+                        int8_t* o = p.rq_codes + (n0 + c * 32) * p.ld_codes + m;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < jmax) {
+                                const float y = __fmul_rn(__int2float_rn((int)v[j] >> shift), scale);
+                                o[(int64_t)j * p.ld_codes] = (int8_t)act_code_exact(y, p.rq_alpha, p.rq_kind, rq_fast);
+                            }
+                        }
+                    }
+                } else if (cfg.tma_store) {
                     const bool tail = cfg.tail_rows && (c == (cfg.npix >> 5));
                     const int nsub = p.acc ? 2 : 1;
                     for (int sub = 0; sub < nsub; ++sub) {
@@ -1014,8 +1045,28 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
             return RMSMP_ERR_CUDA;
     }
 
-    const bool ld_ok = (p.ld_out % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
+    const bool ld_ok = !p.rq_codes && (p.ld_out % 4 == 0) && (p.out_mn ? p.N % 4 == 0 : p.M % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
                        (!p.acc || (reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
+    if (p.rq_codes) {
+        // re-quantized output: [N][ld_codes] code bytes, boxes of 32 rows (bytes) x 32 pixels
+        if (!c.pre || p.out_mn) return RMSMP_ERR_VARIANT;
+        // bulk stores clip at 16-byte granules of the innermost dimension: a row count that is not a
+        // multiple of 16 bytes would spill into the padding columns, so such outputs take direct stores
+        if (p.M % 16 == 0 && p.ld_codes % 16 == 0 && (reinterpret_cast<uintptr_t>(p.rq_codes) & 15) == 0) {
+            auto make = [&](CUtensorMap* m, int rows) -> bool {
+                const cuuint32_t es[2] = {1, 1};
+                const cuuint64_t gs[1] = {(cuuint64_t)p.ld_codes};
+                const cuuint64_t gd[2] = {(cuuint64_t)p.M, (cuuint64_t)p.N};
+                const cuuint32_t bx[2] = {32u, (cuuint32_t)rows};
+                return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, p.rq_codes, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            };
+            bool ok = make(&mp.rq_full, 32);
+            if (ok && c.tail_rows) ok = make(&mp.rq_tail, c.tail_rows);
+            c.tma_store = ok ? 1 : 0;
+        }
+    }
     if (ld_ok && (!p.out_mn || c.tail_rows == 0)) {
         auto make = [&](CUtensorMap* m, void* base, CUtensorMapDataType dt, int rows) -> bool {
             const cuuint32_t es[2] = {1, 1};
@@ -1040,16 +1091,23 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
 
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(tensor_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
-            cudaFuncSetAttribute(tensor_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tensor_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(tensor_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(tensor_kernel<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(tensor_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
             cudaGetLastError();
             return RMSMP_ERR_CUDA;
         }
         attr_set = true;
     }
     const int grid = (int)std::min<int64_t>(c.ntiles, sm_count());
-    if (c.m2) tensor_kernel<1><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
-    else tensor_kernel<0><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
+    if (p.rq_codes) {
+        if (c.m2) tensor_kernel<1, 1><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
+        else tensor_kernel<0, 1><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
+    } else {
+        if (c.m2) tensor_kernel<1, 0><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
+        else tensor_kernel<0, 0><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
+    }
     if (cudaGetLastError() != cudaSuccess) return RMSMP_ERR_CUDA;
     return RMSMP_OK;
 }

@@ -286,3 +286,122 @@ def test_full_path_fp32_in_fp32_out():
     assert np.float32(step) == st_ref
     _, _, _, y_ref = O.layer_conv(Wt, scheme, bits, alpha, codes, st_ref, 1, 1)
     assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.reshape(N, L.M).view(np.uint32))
+
+
+# ------------------------------------------------------------------ re-quantizing epilogue (layer chaining)
+# The fused epilogue must give the codes of (this layer's fp32 output -> the activation quantizer),
+# i.e. the oracle's layer followed by the oracle's quantizer, byte for byte.
+
+def _next_alpha(y_ref):
+    return float(np.float32(3.0 * float(np.std(y_ref))))
+
+
+@pytest.mark.parametrize("kind", [R.ACT_U4, R.ACT_S4])
+@pytest.mark.parametrize("M,K,N,ld_extra", [
+    (256, 512, 300, 0),      # bulk stores, ragged last tile
+    (200, 128, 77, 0),       # ld_codes = 200: not a multiple of 16 -> direct byte stores
+    (130, 96, 513, 14),      # padded leading dimension (144), two row blocks, ragged rows
+    (64, 576, 260, 0),       # duplicated rows, resident weights
+])
+def test_linear_requant_epilogue(M, K, N, ld_extra, kind):
+    import torch
+    g = synth.rng(81, M + K + N)
+    Wt = synth.weights_normal(g, (M, K))
+    codes = synth.act_codes_uniform(g, (N, K))
+    act_step = np.float32(0.125)
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    alpha = synth.alpha_rows(Wt)
+    _, _, _, y_ref = O.layer_linear(Wt, scheme, bits, alpha, codes, act_step)
+    na = _next_alpha(y_ref)
+    want, want_step = O.quantize_act(y_ref.reshape(N, M), na, kind)
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    ld = M + ld_extra
+    out = torch.full((N, ld), 99, dtype=torch.int8, device="cuda")
+    step = R.rmsmp_gemm_workspace_requant(layer, d_packed, ws, torch.from_numpy(codes).cuda(), N, K, float(act_step),
+                                          na, kind, out, ld)
+    torch.cuda.synchronize()
+    assert R.rmsmp_last_device_status(d_packed) == R.OK
+    got = out.cpu().numpy()
+    assert np.float32(step) == want_step
+    assert np.array_equal(got[:, :M], want)
+    assert (got[:, M:] == 99).all()                      # padding columns untouched
+
+
+@pytest.mark.parametrize("kind", [R.ACT_U4, R.ACT_S4])
+@pytest.mark.parametrize("M,Cin,k,stride,pad,B,H,W", [
+    (64, 64, 3, 1, 1, 2, 14, 14),
+    (140, 256, 3, 1, 1, 5, 7, 7),      # several images per tile, ragged last tile, two row blocks
+    (32, 48, 3, 2, 1, 2, 9, 12),
+    (128, 64, 1, 2, 0, 2, 8, 8),
+])
+def test_conv_requant_epilogue(M, Cin, k, stride, pad, B, H, W, kind):
+    import torch
+    g = synth.rng(82, M + Cin + H)
+    Wt = synth.weights_kaiming(g, M, Cin, k, k)
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    alpha = synth.alpha_rows(Wt)
+    x = synth.act_halfnormal(g, (B, H, W, Cin))
+    codes, act_step = O.quantize_act(x, synth.ALPHA_ACT, O.ACT_U4)
+    _, _, _, y_ref = O.layer_conv(Wt, scheme, bits, alpha, codes, act_step, stride, pad)
+    y_ref = y_ref.reshape(-1, M)
+    na = _next_alpha(y_ref)
+    want, want_step = O.quantize_act(y_ref, na, kind)
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    out = torch.full(y_ref.shape, 99, dtype=torch.int8, device="cuda")
+    step = R.rmsmp_conv_implicit_workspace_requant(layer, d_packed, ws, torch.from_numpy(codes).cuda(), B, H, W,
+                                                   stride, pad, float(act_step), na, kind, out)
+    torch.cuda.synchronize()
+    assert R.rmsmp_last_device_status(d_packed) == R.OK
+    assert np.float32(step) == want_step
+    assert np.array_equal(out.cpu().numpy(), want)
+
+
+def test_requant_rejects_bad_arguments():
+    import torch
+    g = synth.rng(83)
+    Wt = synth.weights_normal(g, (32, 64))
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, synth.alpha_rows(Wt))
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    act = torch.zeros((40, 64), dtype=torch.int8, device="cuda")
+    out = torch.zeros((40, 32), dtype=torch.int8, device="cuda")
+    for bad_alpha in (0.0, -1.0, float("inf"), float("nan")):
+        with pytest.raises(R.RmsmpError) as e:
+            R.rmsmp_gemm_workspace_requant(layer, d_packed, ws, act, 40, 64, 0.1, bad_alpha, R.ACT_U4, out, 32)
+        assert e.value.status == R.ERR_SCALE
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_workspace_requant(layer, d_packed, ws, act, 40, 64, 0.1, 1.0, 7, out, 32)
+    assert e.value.status == R.ERR_SCHEME
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_workspace_requant(layer, d_packed, ws, act, 40, 64, 0.1, 1.0, R.ACT_U4, out, 16)   # ld < M
+    assert e.value.status == R.ERR_SHAPE
+
+
+def test_padded_output_rows_leave_the_padding_untouched():
+    """[N][ld_out] fp32 output with ld_out > M and M not a multiple of 4: bulk stores clip in
+    16-byte granules, so this shape must not go through them."""
+    import torch
+    M, K, N, ld = 130, 128, 300, 136
+    g = synth.rng(84)
+    Wt = synth.weights_normal(g, (M, K))
+    codes = synth.act_codes_uniform(g, (N, K))
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    alpha = synth.alpha_rows(Wt)
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    d_codes = torch.from_numpy(codes).cuda()
+    _, _, _, y_ref = O.layer_linear(Wt, scheme, bits, alpha, codes, np.float32(0.25))
+    for fn in (lambda y: R.rmsmp_gemm_workspace(layer, d_packed, ws, d_codes, N, K, 0.25, y, ld),
+               lambda y: R.rmsmp_gemm(layer, d_packed, d_codes, N, K, 0.25, y, ld)):
+        y = torch.full((N, ld), -7.0, dtype=torch.float32, device="cuda")
+        fn(y)
+        torch.cuda.synchronize()
+        got = y.cpu().numpy()
+        assert np.array_equal(got[:, :M].view(np.uint32), y_ref.reshape(N, M).view(np.uint32))
+        assert (got[:, M:] == -7.0).all()

@@ -127,6 +127,14 @@ def test_two_row_blocks_per_tile_full():
     acc_ref = O.matmul(v_ref, c_ref)
     assert np.array_equal(acc.cpu().numpy(), acc_ref)
     assert np.array_equal(y.cpu().numpy().view(np.uint32), _expected(acc_ref, wstep, step).view(np.uint32))
+    # the same shape through the re-quantizing epilogue (next layer's signed 4-bit codes)
+    y_ref = _expected(acc_ref, wstep, step)
+    na = float(np.float32(3.0 * float(np.std(y_ref))))
+    want, _ = O.quantize_act(y_ref, na, O.ACT_S4)
+    out = torch.empty((N, M), dtype=torch.int8, device="cuda")
+    R.rmsmp_gemm_workspace_requant(layer, d_packed, ws, codes, N, K, float(step), na, R.ACT_S4, out, M)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), want)
 
 
 # ------------------------------------------------------------------ config 4: the ResNet-18 stack
