@@ -454,8 +454,8 @@ def run_suite(args):
         R.rmsmp_expand_weights(lay, pk, ws)
         return lay, pk, ws
 
-    VAR = (("tensor_smem", R.VARIANT_TENSOR), ("tensor_workspace", "ws"), ("simt_dp4a", R.VARIANT_SIMT),
-           ("shift_add", R.VARIANT_SHIFTADD))
+    VAR = (("tensor_smem", R.VARIANT_TENSOR), ("tensor_workspace", "ws"), ("workspace_requant", "rq"),
+           ("simt_dp4a", R.VARIANT_SIMT), ("shift_add", R.VARIANT_SHIFTADD))
 
     def bench_shape(cfg, name, M, Cin, k, stride, pad, B, H, ratio=RATIO, pool=1, only=None, iters=20):
         conv = k > 1 or H > 1
@@ -464,6 +464,7 @@ def run_suite(args):
         N = B * Ho * Ho
         act = torch.randint(0, 16, (B, H, H, Cin), dtype=torch.int8, device="cuda")
         y = torch.empty((N, M), dtype=torch.float32, device="cuda")
+        yc = torch.empty((N, M), dtype=torch.int8, device="cuda")
         lay0 = inst[0][0]
         ops = 2 * M * Cin * k * k * N
         pix_in = Ho * Ho if (k == 1 and stride > 1) else H * H
@@ -473,18 +474,21 @@ def run_suite(args):
                 continue
             def fn(i, v=v):
                 lay, pk, ws = inst[i % pool]
-                if v == "ws":
+                if v == "rq":
+                    R.rmsmp_conv_implicit_workspace_requant(lay, pk, ws, act, B, H, H, stride, pad, 0.1, 50.0, R.ACT_U4, yc)
+                elif v == "ws":
                     R.rmsmp_conv_implicit_workspace(lay, pk, ws, act, B, H, H, stride, pad, 0.1, y, R.OUT_NM, None)
                 else:
                     R.rmsmp_conv_implicit_variant(lay, pk, act, B, H, H, stride, pad, 0.1, y, R.OUT_NM, None, v)
             try:
-                us = timed(fn, iters if v in ("ws", R.VARIANT_TENSOR) or ops < 2e10 else 3)
+                us = timed(fn, iters if v in ("ws", "rq", R.VARIANT_TENSOR) or ops < 2e10 else 3)
             except R.RmsmpError as e:
                 print(json.dumps({"suite": cfg, "shape": name, "variant": vname, "error": str(e)}))
                 continue
+            alg_v = alg - 3 * N * M if v == "rq" else alg          # one code byte per output instead of four
             rec = {"suite": cfg, "shape": name, "M": M, "K": Cin * k * k, "N": N, "ratio": list(ratio), "variant": vname,
-                   "us": us, "tops": ops / us / 1e6, "gbs": alg / us / 1e3, "frac_int8_peak": ops / us / 1e6 / i8_peak,
-                   "frac_hbm": alg / us / 1e3 / peaks["hbm_gbs"], "weights": "cold pool of %d" % pool if pool > 1 else "warm"}
+                   "us": us, "tops": ops / us / 1e6, "gbs": alg_v / us / 1e3, "frac_int8_peak": ops / us / 1e6 / i8_peak,
+                   "frac_hbm": alg_v / us / 1e3 / peaks["hbm_gbs"], "weights": "cold pool of %d" % pool if pool > 1 else "warm"}
             rows.append(rec)
             print(json.dumps(rec))
 

@@ -32,7 +32,10 @@ __device__ __forceinline__ ActFast act_fast_setup(float alpha, int kind)
     return f;
 }
 
-// Code of x in the low byte of the result; sets `redo` when the division has to decide.
+// Code of x in the low byte of the result; sets `redo` when the division has to decide: the scaled
+// value here and the one the definition forms differ by a few roundings of relative size 2^-24
+// (< 1e-5 absolute at Q = 15), so they round to the same integer whenever this one is further
+// than 1e-4 from a rounding boundary k + 0.5.
 __device__ __forceinline__ uint32_t act_code_fast(float x, const ActFast& f, bool& redo)
 {
     const float kMagic = 12582912.0f;                       // 1.5 * 2^23: adding it rounds to an integer, half to even
@@ -41,7 +44,7 @@ __device__ __forceinline__ uint32_t act_code_fast(float x, const ActFast& f, boo
     const float u = __fmul_rn(t, f.q);
     const float s = __fadd_rn(u, kMagic);
     const float c = __fsub_rn(s, kMagic);
-    redo = redo || !(fabsf(__fsub_rn(u, c)) <= 0.499f);       // also true for NaN
+    redo = redo || !(fabsf(__fsub_rn(u, c)) <= 0.4999f);      // also true for NaN
     return __float_as_uint(s);                               // low byte = the integer, two's complement
 }
 
@@ -50,8 +53,9 @@ __device__ __forceinline__ uint32_t act_code_fast(float x, const ActFast& f, boo
 __device__ __forceinline__ uint32_t act_code_exact(float x, float alpha, int kind, const ActFast& f)
 {
     bool redo = !f.ok;
-    const uint32_t c = act_code_fast(x, f, redo);
-    return redo ? (uint32_t)act_code(x, alpha, kind) : c;
+    uint32_t c = act_code_fast(x, f, redo);
+    if (redo) c = (uint32_t)act_code(x, alpha, kind);
+    return c;
 }
 
 }  // namespace rmsmp

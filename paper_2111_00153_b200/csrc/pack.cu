@@ -280,7 +280,7 @@ cudaError_t launch_expand(const rmsmp_layer& L, const uint8_t* blob, int8_t* wex
 // Pure streaming kernel.  The code is rint(clip(x / alpha) * Q) with ONE correctly rounded fp32
 // division; that division costs more issue slots than the memory system leaves time for, so the
 // vector path first forms the code from x * (1 / alpha) and keeps it only when the scaled value
-// is not within 0.001 of a rounding boundary (k + 0.5), where the two ways of computing x / alpha
+// is not within 1e-4 of a rounding boundary (k + 0.5), where the two ways of computing x / alpha
 // (relative difference < 2^-22) cannot round to different integers; the few values that are
 // close to a boundary, and NaNs, take the division.  The results are those of act_code() in
 // every case.
