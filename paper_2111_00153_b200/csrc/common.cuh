@@ -75,6 +75,9 @@ cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t t
 // returns false if the tensor variant cannot run this problem (alignment / shape)
 bool tensor_supported(const Problem& p);
 rmsmp_status launch_tensor(const Problem& p, cudaStream_t st);
+// two-CTA form of the workspace mode (tensor2.cu): false if it cannot, or should not, run this problem
+bool pair_supported(const Problem& p);
+rmsmp_status launch_pair(const Problem& p, cudaStream_t st);
 
 // ---- device helpers used by more than one kernel file ----
 

@@ -1015,6 +1015,7 @@ bool tensor_supported(const Problem& p)
 
 rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
 {
+    if (pair_supported(p)) return launch_pair(p, st);
     TensorCfg c;
     if (!plan(p, c)) return RMSMP_ERR_VARIANT;
     EncodeTiledFn enc = encode_fn();

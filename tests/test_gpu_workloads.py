@@ -239,3 +239,56 @@ def test_config5_grouped_launch_matches_oracle(N):
     for (layer, d_packed, a, y, acc), (acc_ref, y_ref) in zip(keep, refs):
         assert np.array_equal(acc.cpu().numpy(), acc_ref)
         assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
+
+
+# ------------------------------------------------------------------ CTA-pair kernel (long K, even row blocks, fp32 [N][M] output)
+
+@pytest.mark.parametrize("M,K,N", [
+    (256, 2048, 1000),      # ragged last half (1000 = 7 * 128 + 104), odd number of halves
+    (500, 2304, 300),       # four row blocks, the last one ragged; last tile has one empty half
+    (512, 4096, 129),       # second half holds a single token
+])
+def test_cta_pair_linear_full(M, K, N):
+    """Shapes that run on the two-CTA kernel when called without an accumulator dump; the same call
+    with a dump runs on the single-CTA kernel.  Both against the oracle, element by element."""
+    import torch
+    g = synth.rng(3, M + K + N)
+    W = synth.weights_normal(g, (M, K))
+    c_ref = synth.act_codes_uniform(g, (N, K))
+    step = np.float32(0.0625)
+    scheme, bits = O.assign_rows(W, synth.RATIO_RMSMP1)
+    alpha = synth.alpha_rows(W)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    codes = torch.from_numpy(c_ref).cuda()
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    y_pair = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+    R.rmsmp_gemm_workspace(layer, d_packed, ws, codes, N, K, float(step), y_pair, M)
+    y_one = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+    acc = torch.empty((N, M), dtype=torch.int32, device="cuda")
+    R.rmsmp_gemm_workspace(layer, d_packed, ws, codes, N, K, float(step), y_one, M, R.OUT_NM, acc)
+    torch.cuda.synchronize()
+    assert R.rmsmp_last_device_status(d_packed) == R.OK
+    v_ref, wstep = O.quantize_rows(W, scheme, bits, alpha)
+    acc_ref = O.matmul(v_ref, c_ref)
+    want = _expected(acc_ref, wstep, step)
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    assert np.array_equal(y_one.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    assert np.array_equal(y_pair.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("M,Cin,k,stride,pad,B,H", [
+    (256, 256, 3, 1, 1, 5, 14),      # halves of 7 rows; 10 halves
+    (256, 256, 3, 2, 1, 3, 28),      # stride 2: 14x14 outputs
+    (512, 512, 3, 1, 1, 7, 7),       # two images per half, odd image count
+    (256, 128, 5, 1, 2, 2, 20),      # 5x5 taps (25 k-blocks), halves of 5 rows of 20 pixels
+])
+def test_cta_pair_conv_full(M, Cin, k, stride, pad, B, H):
+    g = synth.rng(4, M + Cin + k + H)
+    W = synth.weights_kaiming(g, M, Cin, k, k)
+    x = synth.act_halfnormal(g, (B, H, H, Cin))
+    scheme, bits = R.rmsmp_assign_rows(W, synth.RATIO_RMSMP1)
+    alpha = synth.alpha_rows(W)
+    codes, step, y = _run_conv_device(W, scheme, bits, alpha, x, stride, pad, R.ACT_U4)
+    _, ws, acc, y_ref = O.layer_conv(W, scheme, bits, alpha, codes, step, stride, pad)
+    assert np.array_equal(y.view(np.uint32), y_ref.reshape(-1, M).view(np.uint32))
