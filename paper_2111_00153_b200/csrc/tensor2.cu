@@ -10,7 +10,7 @@
 // Roles per CTA (448 threads): warp 0 lane 0 fetches this CTA's half of the activation codes,
 // warp 2 lane 0 its 128 expanded weight rows (both signal the LEADER's "full" barrier, rank 0;
 // warps 3 and 4 are second producers taking the odd k-blocks),
-// warp 1 of the leader issues the MMAs and commits to both CTAs' barriers, warps 5-13 are the
+// warp 1 of the leader issues the MMAs and commits to both CTAs' barriers, warps 6-13 are the
 // epilogue of this CTA's 128 rows (tcgen05.ld, scale, staged bulk stores as in the single-CTA
 // kernel).  Accumulators: tensor-memory columns [0, N) and [256, 256 + N), alternating by tile.
 // A tile's pixels are two "halves" of up to 128 pixels each (whole images, or whole output rows of
@@ -32,9 +32,10 @@ constexpr int kThreads2 = 448;
 constexpr int kStageA = 128 * 128;               // 16 KB: 128 rows x 128 B
 constexpr int kStageB = 128 * 128;               // 16 KB: up to 128 pixels x 128 B
 constexpr int kWarpStage2 = 32 * 32 * 4;         // per-warp output staging
-constexpr int kEpiWarps2 = 9;
-constexpr int kFirstEpi2 = 5;                   // warps 5-13
-constexpr int kRing2 = 5;
+constexpr int kEpiWarps2 = 8;
+constexpr int kFirstEpi2 = 6;                   // warps 6-13, two per tensor-memory quarter
+constexpr int kRing2 = 3;                       // stages; a stage holds TWO k-blocks of each operand (64 KB per CTA)
+constexpr int kSub2 = 2;
 constexpr long long kWaitCycles2 = 2000000000LL;
 
 struct PairCfg {
@@ -197,8 +198,8 @@ pair_kernel(const Problem p, const PairCfg cfg, const __grid_constant__ PairMaps
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (s32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sA = smem_base;
-    const uint32_t sB = sA + kRing2 * kStageA;
-    const uint32_t sOut = sB + kRing2 * kStageB;
+    const uint32_t sB = sA + kRing2 * kSub2 * kStageA;
+    const uint32_t sOut = sB + kRing2 * kSub2 * kStageB;
     const uint32_t sBar = sOut + kEpiWarps2 * kWarpStage2;
     const uint32_t bar_full = sBar, bar_empty = sBar + 8 * kRing2;
     const uint32_t bar_tfull = sBar + 16 * kRing2, bar_tempty = bar_tfull + 16;
@@ -239,7 +240,7 @@ pair_kernel(const Problem p, const PairCfg cfg, const __grid_constant__ PairMaps
       if (lane == 0) {
         // ---------------------------------------------------------- producers (both CTAs)
         // One thread can start a bulk tensor copy only every ~300 ns, about the time four MMAs take,
-        // so each operand has two producer threads taking alternate k-blocks.
+        // so each operand has two producer threads taking alternate stages.
         const bool is_b = (warp == 0 || warp == 3);
         const uint32_t mine = (warp >= 3) ? 1u : 0u;
         uint32_t s = 0, ph = 0, g = 0;
@@ -250,24 +251,25 @@ pair_kernel(const Problem p, const PairCfg cfg, const __grid_constant__ PairMaps
             const HalfPos hp = half_pos(p, cfg, 2 * nt + rank);               // this CTA's half of the pixels
             const int y_base = hp.h0 * p.stride - p.pad;
             int tap = 0, cc = 0, ti = 0, tj = 0;
-            for (int kb = 0; kb < cfg.nkb; ++kb, ++g) {
-                if ((g & 1u) != mine) {
-                    if (++s == kRing2) { s = 0; ph ^= 1; }
-                    if (++cc == cfg.cpt) { cc = 0; ++tap; if (++tj == p.kw) { tj = 0; ++ti; } }
-                    continue;
+            for (int kb = 0; kb < cfg.nkb; kb += kSub2, ++g) {
+                const int nsub = min(kSub2, cfg.nkb - kb);
+                const bool skip = (g & 1u) != mine;
+                if (!skip) {
+                    if (!bar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
+                    // all copies of this stage (up to two k-blocks of two operands in two CTAs) complete on the leader's barrier
+                    if (is_b && rank == 0)
+                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                                     ::"r"(bar_full + 8 * s), "r"(2u * nsub * (cfg.tx_b + (uint32_t)kStageA)) : "memory");
                 }
-                if (!bar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
                 const uint32_t fb = lead_full + 8 * s;
-                if (is_b) {
-                    // all four copies of this k-block (two per CTA) complete on the leader's barrier
-                    if (rank == 0)
-                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_full + 8 * s), "r"(2 * (cfg.tx_b + (uint32_t)kStageA)) : "memory");
-                    pair_load_4d(sB + s * kStageB, &maps.act, fb, cc * 128, tj - p.pad, y_base + ti, hp.b0);
-                } else {
-                    pair_load_2d(sA + s * kStageA, &maps.wexp, fb, tap * p.Cp + cc * 128, blk * kBlockRows);
+                for (int u = 0; u < nsub; ++u) {
+                    if (!skip) {
+                        if (is_b) pair_load_4d(sB + (s * kSub2 + u) * kStageB, &maps.act, fb, cc * 128, tj - p.pad, y_base + ti, hp.b0);
+                        else pair_load_2d(sA + (s * kSub2 + u) * kStageA, &maps.wexp, fb, tap * p.Cp + cc * 128, blk * kBlockRows);
+                    }
+                    if (++cc == cfg.cpt) { cc = 0; ++tap; if (++tj == p.kw) { tj = 0; ++ti; } }
                 }
                 if (++s == kRing2) { s = 0; ph ^= 1; }
-                if (++cc == cfg.cpt) { cc = 0; ++tap; if (++tj == p.kw) { tj = 0; ++ti; } }
             }
         }
         if (!ok) {
@@ -281,7 +283,7 @@ pair_kernel(const Problem p, const PairCfg cfg, const __grid_constant__ PairMaps
             uint32_t s = 0, ph = 0, it = 0;
             const uint32_t hi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);     // SBO 1024 B, version 1, 128-byte swizzle
             const uint32_t a_lo0 = ((sA >> 4) & 0x3FFFu) | (1u << 16), b_lo0 = ((sB >> 4) & 0x3FFFu) | (1u << 16);
-            const uint32_t a_step = kStageA >> 4, b_step = kStageB >> 4;
+            const uint32_t a_step = (kSub2 * kStageA) >> 4, b_step = (kSub2 * kStageB) >> 4;
             uint32_t a_lo = a_lo0, b_lo = b_lo0;
             for (int64_t tile = first; tile < cfg.ntiles && !*abort_flag; tile += step, ++it) {
                 const uint32_t ab = it & 1;
@@ -289,7 +291,7 @@ pair_kernel(const Problem p, const PairCfg cfg, const __grid_constant__ PairMaps
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + ab * 256;
                 bool ok = true;
-                for (int kb = 0; kb < cfg.nkb; ++kb) {
+                for (int kb = 0; kb < cfg.nkb; kb += kSub2) {
                     if (!bar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     if (issuer) {
@@ -297,6 +299,13 @@ pair_kernel(const Problem p, const PairCfg cfg, const __grid_constant__ PairMaps
                         pair_mma(d_tmem, a_lo + 2, b_lo + 2, hi, cfg.idesc, 1u);
                         pair_mma(d_tmem, a_lo + 4, b_lo + 4, hi, cfg.idesc, 1u);
                         pair_mma(d_tmem, a_lo + 6, b_lo + 6, hi, cfg.idesc, 1u);
+                        if (kb + 1 < cfg.nkb) {
+                            const uint32_t a1 = a_lo + (kStageA >> 4), b1 = b_lo + (kStageB >> 4);
+                            pair_mma(d_tmem, a1, b1, hi, cfg.idesc, 1u);
+                            pair_mma(d_tmem, a1 + 2, b1 + 2, hi, cfg.idesc, 1u);
+                            pair_mma(d_tmem, a1 + 4, b1 + 4, hi, cfg.idesc, 1u);
+                            pair_mma(d_tmem, a1 + 6, b1 + 6, hi, cfg.idesc, 1u);
+                        }
                         pair_commit(bar_empty + 8 * s);
                     }
                     a_lo += a_step;
@@ -449,7 +458,7 @@ bool plan_pair(const Problem& p, PairCfg& c)
     c.tail_rows = c.npix_h & 31;
     // kind::i8, int32 accumulate, signed 8-bit A and B, K-major; N = both halves, M = 256 over the pair
     c.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * c.nh_pad) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-    c.smem_bytes = (uint32_t)(kRing2 * (kStageA + kStageB) + kEpiWarps2 * kWarpStage2 + 1024 + 64 * 2 * kRing2);
+    c.smem_bytes = (uint32_t)(kRing2 * kSub2 * (kStageA + kStageB) + kEpiWarps2 * kWarpStage2 + 1024 + 64 * 2 * kRing2);
     return true;
 }
 
