@@ -75,9 +75,41 @@ cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t t
 // returns false if the tensor variant cannot run this problem (alignment / shape)
 bool tensor_supported(const Problem& p);
 rmsmp_status launch_tensor(const Problem& p, cudaStream_t st);
+// fills four CUtensorMap objects (see act_parity_split; only the first is used without the split) for
+// activation boxes of bk channels x th output rows x tb images, swizzle width = bk bytes
+bool encode_act_maps_4(const Problem& p, int bk, int th, int tb, void* maps4);
 // two-CTA form of the workspace mode (tensor2.cu): false if it cannot, or should not, run this problem
 bool pair_supported(const Problem& p);
 rmsmp_status launch_pair(const Problem& p, cudaStream_t st);
+
+// ---- activation boxes of the tensor-core kernels ----
+// A stride-2 convolution reads, for one filter tap, every second pixel of every second input row.
+// Asking the copy engine for that with element strides makes it fetch pixel by pixel (measured: an
+// order of magnitude below its unit-stride rate).  Instead the input is seen as four sub-grids by
+// row and column parity, each with its own tensor map of doubled global strides and unit element
+// strides; the pixels one tap needs for a whole tile lie in ONE sub-grid and form a dense box
+// there.  Out-of-range coordinates of a sub-grid read zeros, which is the padding, as before.
+__host__ __device__ inline bool act_parity_split(const Problem& p)
+{
+    return p.stride == 2 && p.H >= 2 && p.W >= 2;
+}
+struct TapBox { int map, x, y; };      // tensor map index (row parity * 2 + column parity), box start
+__host__ __device__ inline TapBox tap_box(const Problem& p, int h0, int ti, int tj)
+{
+    TapBox t;
+    const int dy = ti - p.pad, dx = tj - p.pad;
+    if (act_parity_split(p)) {
+        const int py = dy & 1, px = dx & 1;            // two's complement: -1 & 1 == 1
+        t.map = py * 2 + px;
+        t.y = h0 + ((dy - py) >> 1);                   // dy - py is even; arithmetic shift
+        t.x = (dx - px) >> 1;
+    } else {
+        t.map = 0;
+        t.y = h0 * p.stride + dy;
+        t.x = dx;
+    }
+    return t;
+}
 
 // ---- device helpers used by more than one kernel file ----
 

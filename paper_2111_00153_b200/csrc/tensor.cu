@@ -64,6 +64,10 @@ struct TensorCfg {
     int nA, nB, nR;        // ring depths: expanded weights, activations, raw weights
     uint32_t raw_bytes;    // one raw stage
     int out_bufs;          // staging buffers per epilogue warp (1 or 2)
+    int fastcvt;           // 1: every |accumulator| of this problem is below 2^22, so int -> float is done exactly with
+                           //    an integer add and a float subtract (see acc_to_float_small) instead of a conversion
+                           //    instruction, whose pipe runs at a fraction of the arithmetic rate and bounds the
+                           //    epilogue of output-bound layers
     int pre;               // 1: the A operand comes expanded (int8) from a workspace, no expander work
     int dup;               // 1 (pre mode, M <= 64): rows 0..63 are loaded twice, into lanes 0..63 and 64..127, so that all
                            //    four tensor-memory quarters hold valid rows and every epilogue warp has work
@@ -80,11 +84,15 @@ struct TensorCfg {
     int tps;               // k-blocks per activation stage: 1, or 3 (resident weights, 64-byte k-blocks, 3-wide kernels):
                            //    one barrier round trip then covers a whole kernel row instead of a single tap
     int b_sub;             // bytes of one k-block inside an activation stage
+    int colshift;          // 1 (with tps == 3; 3x3, stride 1, tiles of whole output rows of one image, W % 8 == 0): an activation
+                           //    stage holds the th + 2 input rows the tile needs at ONE column shift j, fetched once; the
+                           //    taps (0..2, j) read it at row offsets of W pixels (whole swizzle atoms).  The copy engine
+                           //    then moves 3 (th + 2) rows per tile instead of 9 th
     uint32_t smem_bytes;
 };
 
 struct Maps {
-    CUtensorMap act;                                   // [B][H][W][Cin] activation codes
+    CUtensorMap act[4];                                // [B][H][W][Cin] activation codes; stride 2: one map per row/column parity
     CUtensorMap q4, q8;                                // packed weight regions
     CUtensorMap wexp;                                  // [M][Kp] int8 weights expanded beforehand (pre mode); 64-row box when dup
     CUtensorMap out_full, out_tail, acc_full, acc_tail;   // bulk stores: 32-row and tail chunks
@@ -227,6 +235,14 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32])
                  :: "memory");
 }
 
+// Exact float value of an integer |a| < 2^22 without a conversion instruction: the bit pattern of
+// 1.5 * 2^23 plus a is the float 12582912 + a (floats in [2^23, 2^24) are the integers), and
+// subtracting 12582912 back is exact.
+__device__ __forceinline__ float acc_to_float_small(int a)
+{
+    return __fsub_rn(__int_as_float(a + 0x4B400000), 12582912.0f);
+}
+
 // ------------------------------------------------------------------ per-tile row bookkeeping
 
 // Rows of one 128-row block inside the three groups of the packed buffer.
@@ -365,21 +381,34 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
             uint32_t s = 0, ph = 0;
             bool ok = true;
             for (int64_t tile = first; tile < cfg.ntiles && ok; tile += step) {
-                const int64_t nt = tile / cfg.nbt;
-                const int blk = (int)(tile - nt * cfg.nbt) << kM2;
+                const uint32_t nt = (uint32_t)tile / (uint32_t)cfg.nbt;
+                const int blk = (int)((uint32_t)tile - nt * (uint32_t)cfg.nbt) << kM2;
                 int b0, h0;
-                if (cfg.tiles_per_image) { b0 = (int)(nt / cfg.tiles_per_image); h0 = (int)(nt % cfg.tiles_per_image) * cfg.th; }
-                else { b0 = (int)(nt * cfg.tb); h0 = 0; }
+                if (cfg.tiles_per_image) {
+                    b0 = (int)(nt / (uint32_t)cfg.tiles_per_image);
+                    h0 = (int)(nt - (uint32_t)b0 * (uint32_t)cfg.tiles_per_image) * cfg.th;
+                } else {
+                    b0 = (int)nt * cfg.tb;
+                    h0 = 0;
+                }
                 const int row_a = cfg.dup ? 0 : blk * kBlockRows;
-                const int y_base = h0 * p.stride - p.pad;
                 int tap = 0, cc = 0, ti = 0, tj = 0;
                 for (int kb = 0; kb < cfg.nkb; ++kb) {
                     if (!mbar_wait(bar_e + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
                     if (pre_b_producer && cfg.tps > 1) {
-                        // one stage = the taps of one kernel row (one channel chunk per tap in this mode)
-                        mbar_arrive_expect_tx(bar_f + 8 * s, cfg.tps * cfg.tx_bytes);
-                        for (int t = 0; t < cfg.tps; ++t)
-                            tma_load_4d(sB + s * cfg.b_bytes + t * cfg.b_sub, &maps.act, bar_f + 8 * s, 0, tj + t - p.pad, y_base + ti, b0);
+                        if (cfg.colshift) {
+                            // one stage = one column shift: the th + kh - 1 input rows the tile needs, fetched once
+                            // and read by the kh taps of that column at row offsets (see TensorCfg::colshift)
+                            mbar_arrive_expect_tx(bar_f + 8 * s, cfg.tx_bytes);
+                            tma_load_4d(sB + s * cfg.b_bytes, &maps.act[0], bar_f + 8 * s, 0, ti - p.pad, h0 - p.pad, b0);
+                        } else {
+                            // one stage = the taps of one kernel row (one channel chunk per tap in this mode)
+                            mbar_arrive_expect_tx(bar_f + 8 * s, cfg.tps * cfg.tx_bytes);
+                            for (int t = 0; t < cfg.tps; ++t) {
+                                const TapBox tb = tap_box(p, h0, ti, tj + t);
+                                tma_load_4d(sB + s * cfg.b_bytes + t * cfg.b_sub, &maps.act[tb.map], bar_f + 8 * s, 0, tb.x, tb.y, b0);
+                            }
+                        }
                         ++ti;
                         kb += cfg.tps - 1;
                         if (++s == nring) { s = 0; ph ^= 1; }
@@ -387,7 +416,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                     }
                     if (pre_b_producer) {
                         mbar_arrive_expect_tx(bar_f + 8 * s, cfg.tx_bytes);
-                        tma_load_4d(sB + s * cfg.b_bytes, &maps.act, bar_f + 8 * s, cc * cfg.bk, tj - p.pad, y_base + ti, b0);
+                        const TapBox tb = tap_box(p, h0, ti, tj);
+                        tma_load_4d(sB + s * cfg.b_bytes, &maps.act[tb.map], bar_f + 8 * s, cc * cfg.bk, tb.x, tb.y, b0);
                     } else {
                         const int koff = tap * p.Cp + cc * cfg.bk;
                         mbar_arrive_expect_tx(bar_f + 8 * s, cfg.a_bytes);
@@ -477,8 +507,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                     if (lane == 0) {
                         const int ti = tap / p.kw, tj = tap - ti * p.kw;
                         mbar_arrive_expect_tx(bar_fullB + 8 * sb, cfg.tx_bytes);
-                        tma_load_4d(sB + sb * cfg.b_bytes, &maps.act, bar_fullB + 8 * sb, c0, tj - p.pad,
-                                    h0 * p.stride + ti - p.pad, b0);
+                        const TapBox tb = tap_box(p, h0, ti, tj);
+                        tma_load_4d(sB + sb * cfg.b_bytes, &maps.act[tb.map], bar_fullB + 8 * sb, c0, tb.x, tb.y, b0);
                     }
                     if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; }
                     if (++cc == cfg.cpt) { cc = 0; ++tap; }
@@ -509,9 +539,13 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 bool ok = true;
                 int cc = 0;
                 if (cfg.tps > 1) {
-                    // resident weights, three 64-byte k-blocks per activation stage (never with two row blocks)
-                    const uint32_t a_step = (uint32_t)cfg.a_bytes >> 4, b_step = (uint32_t)cfg.b_bytes >> 4,
-                                   t_step = (uint32_t)cfg.b_sub >> 4;
+                    // resident weights, three 64-byte k-blocks per activation stage (never with two row blocks):
+                    // the taps of a kernel row in three sub-buffers, or (colshift) the taps of a kernel COLUMN
+                    // reading one buffer at three row offsets
+                    const uint32_t a_step = (uint32_t)cfg.a_bytes >> 4, b_step = (uint32_t)cfg.b_bytes >> 4;
+                    const uint32_t t_step = cfg.colshift ? ((uint32_t)(p.W * cfg.bk) >> 4) : ((uint32_t)cfg.b_sub >> 4);
+                    const uint32_t a_t = cfg.colshift ? 3 * a_step : a_step;       // between the three MMAs of a stage
+                    const uint32_t a_adv = cfg.colshift ? a_step : 3 * a_step;     // from stage to stage
                     uint32_t a_lo = desc_lo0_a, b_lo = desc_lo0_b + sb * b_step;
                     const bool two = (cfg.last_ksteps == 2);
                     for (int kb = 0; kb < cfg.nkb; kb += 3) {
@@ -520,13 +554,13 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                         if (issuer) {
                             mma_i8_halves(d_tmem, a_lo, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
                             if (two) mma_i8_halves(d_tmem, a_lo + 2, b_lo + 2, desc_hi, cfg.idesc, 1u);
-                            mma_i8_halves(d_tmem, a_lo + a_step, b_lo + t_step, desc_hi, cfg.idesc, 1u);
-                            if (two) mma_i8_halves(d_tmem, a_lo + a_step + 2, b_lo + t_step + 2, desc_hi, cfg.idesc, 1u);
-                            mma_i8_halves(d_tmem, a_lo + 2 * a_step, b_lo + 2 * t_step, desc_hi, cfg.idesc, 1u);
-                            if (two) mma_i8_halves(d_tmem, a_lo + 2 * a_step + 2, b_lo + 2 * t_step + 2, desc_hi, cfg.idesc, 1u);
+                            mma_i8_halves(d_tmem, a_lo + a_t, b_lo + t_step, desc_hi, cfg.idesc, 1u);
+                            if (two) mma_i8_halves(d_tmem, a_lo + a_t + 2, b_lo + t_step + 2, desc_hi, cfg.idesc, 1u);
+                            mma_i8_halves(d_tmem, a_lo + 2 * a_t, b_lo + 2 * t_step, desc_hi, cfg.idesc, 1u);
+                            if (two) mma_i8_halves(d_tmem, a_lo + 2 * a_t + 2, b_lo + 2 * t_step + 2, desc_hi, cfg.idesc, 1u);
                             mma_commit(bar_emptyB + 8 * sb);
                         }
-                        a_lo += 3 * a_step;
+                        a_lo += a_adv;
                         b_lo += b_step;
                         if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; b_lo = desc_lo0_b; }
                     }
@@ -679,25 +713,37 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         const uint32_t my_stage = sOut + (uint32_t)ew * (cfg.out_bufs * kWarpStage);
         uint32_t it = 0, stg_count = 0;
         bool alive = true;
+        int scale_blk = -1, shift = 0;
+        float scale = 0.f;
         const ActFast rq_fast = act_fast_setup(kRQ ? p.rq_alpha : 1.0f, kRQ ? p.rq_kind : 0);
         for (int64_t tile = first; tile < cfg.ntiles && alive; tile += step, ++it) {
           // a tile is one row block (accumulators alternate between tiles), or two (one accumulator each)
           for (int half = 0; half <= kM2; ++half) {
             const uint32_t ab = kM2 ? (uint32_t)half : (it & 1);
             const uint32_t tpar = kM2 ? (it & 1) : ((it >> 1) & 1);
-            const int64_t nt = tile / cfg.nbt;
-            const int blk = ((int)(tile - nt * cfg.nbt) << kM2) + half;
+            // tile indices fit 32 bits (checked on the host): 32-bit divisions, a fraction of the 64-bit ones' cost,
+            // which every epilogue warp would otherwise pay in front of each tile
+            const uint32_t nt = (uint32_t)tile / (uint32_t)cfg.nbt;
+            const int blk = ((int)((uint32_t)tile - nt * (uint32_t)cfg.nbt) << kM2) + half;
             int64_t n0;
-            if (cfg.tiles_per_image) n0 = ((nt / cfg.tiles_per_image) * p.Ho + (nt % cfg.tiles_per_image) * cfg.th) * (int64_t)p.Wo;
-            else n0 = nt * (int64_t)cfg.npix;
+            if (cfg.tiles_per_image) {
+                const uint32_t img = nt / (uint32_t)cfg.tiles_per_image, tin = nt - img * (uint32_t)cfg.tiles_per_image;
+                n0 = ((int64_t)img * p.Ho + (int64_t)tin * cfg.th) * (int64_t)p.Wo;
+            } else {
+                n0 = (int64_t)nt * cfg.npix;
+            }
             const int nvalid = (int)min((int64_t)cfg.npix, p.N - n0);
             const int m = blk * kBlockRows + row0 + lane;
             const bool row_ok = m < p.M;
-            float scale = 0.f;
-            int shift = 0;
-            if (row_ok) {
-                scale = __fmul_rn(__ldg(p.wstep + m), p.act_step);
-                shift = (!cfg.pre && __ldg(p.kind + m) == kFixed4) ? 4 : 0;   // expanders store Fixed-4 codes as 16 * value
+            if (blk != scale_blk) {
+                // the row's scale: loaded when the row block changes (never again for layers of one row block)
+                scale_blk = blk;
+                scale = 0.f;
+                shift = 0;
+                if (row_ok) {
+                    scale = __fmul_rn(__ldg(p.wstep + m), p.act_step);
+                    shift = (!cfg.pre && __ldg(p.kind + m) == kFixed4) ? 4 : 0;   // expanders store Fixed-4 codes as 16 * value
+                }
             }
             if (!mbar_wait_warp(bar_tfull + 8 * ab, tpar, abort_flag)) { alive = false; break; }
             tc_fence_after();
@@ -779,11 +825,19 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                         if (!p.out_mn) {
                             // [pixel][row]: the warp writes 128 contiguous bytes per pixel
                             const uint32_t a0 = stg + lane * 4;
+                            if (cfg.fastcvt && !sub) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const int a = (int)v[j] >> shift;
-                                const uint32_t w = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
-                                asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 128), "r"(w) : "memory");
+                                for (int j = 0; j < 32; ++j) {
+                                    const uint32_t w = __float_as_uint(__fmul_rn(acc_to_float_small((int)v[j] >> shift), scale));
+                                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 128), "r"(w) : "memory");
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) {
+                                    const int a = (int)v[j] >> shift;
+                                    const uint32_t w = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
+                                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 128), "r"(w) : "memory");
+                                }
                             }
                         } else {
                             // [row][pixel], 16-byte chunks swizzled by row (matches the 128-byte-swizzled store map)
@@ -904,6 +958,35 @@ int sm_count()
     return n;
 }
 
+// Tensor maps of the activation codes for boxes of `bk` channels x th output rows x tb images
+// (see act_parity_split: one map, or one per parity sub-grid of a stride-2 layer).
+bool encode_act_maps(EncodeTiledFn enc, const Problem& p, int bk, int th, int tb, CUtensorMapSwizzle swz, CUtensorMap out[4])
+{
+    const cuuint64_t pitch = (cuuint64_t)p.pix_pitch;
+    if (act_parity_split(p)) {
+        for (int py = 0; py < 2; ++py)
+            for (int px = 0; px < 2; ++px) {
+                const cuuint64_t gdim[4] = {(cuuint64_t)p.Cin, (cuuint64_t)((p.W - px + 1) / 2), (cuuint64_t)((p.H - py + 1) / 2), (cuuint64_t)p.B};
+                const cuuint64_t gstr[3] = {2 * pitch, 2 * pitch * p.W, pitch * p.W * p.H};
+                const cuuint32_t box[4] = {(cuuint32_t)bk, (cuuint32_t)p.Wo, (cuuint32_t)th, (cuuint32_t)tb};
+                const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+                const int8_t* base = p.act + ((int64_t)py * p.W + px) * p.pix_pitch;
+                if (enc(&out[py * 2 + px], CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(base), gdim, gstr, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                    return false;
+            }
+        return true;
+    }
+    const cuuint64_t gdim[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+    const cuuint64_t gstr[3] = {pitch, pitch * p.W, pitch * p.W * p.H};
+    const cuuint32_t box[4] = {(cuuint32_t)bk, (cuuint32_t)(p.Wo * p.stride), (cuuint32_t)(th * p.stride), (cuuint32_t)tb};
+    const cuuint32_t estr[4] = {1u, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1u};
+    return enc(&out[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(p.act), gdim, gstr, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool plan(const Problem& p, TensorCfg& c)
 {
     if (p.pix_pitch % 16 != 0 || p.Cin % 16 != 0) return false;
@@ -929,10 +1012,12 @@ bool plan(const Problem& p, TensorCfg& c)
     c.npix = c.tb * c.th * p.Wo;
     c.n_mma = (c.npix + 15) / 16 * 16;
     c.ntiles = c.ntiles_n * p.nblocks;
+    if (c.ntiles >= (1ll << 31)) return false;
     c.m2 = 0;
     c.nbt = p.nblocks;
     c.tps = 1;
     c.b_sub = 0;
+    c.colshift = 0;
     c.pre = p.wexp ? 1 : 0;
     // 64-byte k-blocks when a 128-byte row would be at most half used by the (last) channel chunk
     c.bk = (c.pre && (p.Cin % 128 != 0) && (p.Cin % 128 <= 64)) ? 64 : 128;
@@ -947,6 +1032,9 @@ bool plan(const Problem& p, TensorCfg& c)
     c.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.n_mma >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
     c.tail_rows = c.npix & 31;
     c.tma_store = 0;
+    // |acc| <= K * 127 * 15 (4-bit activation codes, 8-bit weights at most), times 16 while Fixed-4 rows are
+    // expanded as 16 * value in shared-memory expansion mode
+    c.fastcvt = ((int64_t)p.kh * p.kw * p.Cin * 127 * 15 * (p.wexp ? 1 : 16) < (1ll << 22)) ? 1 : 0;
     c.dup = 0;
     c.ares = 0;
     c.epi_warps = kNumEpiWarps;
@@ -968,10 +1056,15 @@ bool plan(const Problem& p, TensorCfg& c)
             c.tps = 3;
             c.b_sub = (c.n_mma * c.bk + 1023) / 1024 * 1024;
             c.b_bytes = c.tps * c.b_sub;
+            if (p.kh == 3 && p.stride == 1 && p.Wo == p.W && c.tb == 1 && p.W % 8 == 0 && c.npix == c.th * p.W) {
+                c.colshift = 1;
+                c.tx_bytes = (uint32_t)((c.th + 2) * p.W * c.bk);
+                c.b_bytes = ((c.th + 2) * p.W * c.bk + 1023) / 1024 * 1024;
+            }
             const int64_t left = kSmemLimit - (1024 + 64 * kMaxRing) - (int64_t)c.nkb * c.a_bytes -
                                  (int64_t)c.epi_warps * kWarpStage;
             c.nB = (int)std::min<int64_t>(kMaxRing, left / c.b_bytes);
-            if (c.nB < 2) { c.tps = 1; c.b_bytes = kTileN * c.bk; c.b_sub = c.b_bytes; c.nB = (int)std::min<int64_t>(kMaxRing, left / c.b_bytes); }
+            if (c.nB < 2) { c.tps = 1; c.colshift = 0; c.tx_bytes = (uint32_t)c.npix * (uint32_t)c.bk; c.b_bytes = kTileN * c.bk; c.b_sub = c.b_bytes; c.nB = (int)std::min<int64_t>(kMaxRing, left / c.b_bytes); }
         }
         // Two row blocks per tile pay when K is long (the two accumulators' epilogue is only half
         // hidden behind the next tile's MMAs) and when the halved tile count does not cost more in
@@ -1007,6 +1100,13 @@ bool plan(const Problem& p, TensorCfg& c)
 
 }  // namespace
 
+bool encode_act_maps_4(const Problem& p, int bk, int th, int tb, void* maps4)
+{
+    EncodeTiledFn enc = encode_fn();
+    return enc && encode_act_maps(enc, p, bk, th, tb, bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                                  static_cast<CUtensorMap*>(maps4));
+}
+
 bool tensor_supported(const Problem& p)
 {
     TensorCfg c;
@@ -1022,17 +1122,8 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
     if (!enc) return RMSMP_ERR_CUDA;
     Maps mp;
     memset(&mp, 0, sizeof(mp));
-    {
-        const cuuint64_t gdim[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
-        const cuuint64_t gstr[3] = {(cuuint64_t)p.pix_pitch, (cuuint64_t)p.pix_pitch * p.W,
-                                    (cuuint64_t)p.pix_pitch * p.W * p.H};
-        const cuuint32_t box[4] = {(cuuint32_t)c.bk, (cuuint32_t)(p.Wo * p.stride), (cuuint32_t)(c.th * p.stride), (cuuint32_t)c.tb};
-        const cuuint32_t estr[4] = {1u, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1u};
-        if (enc(&mp.act, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(p.act), gdim, gstr, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, c.bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return RMSMP_ERR_CUDA;
-    }
+    if (!encode_act_maps(enc, p, c.bk, c.colshift ? c.th + 2 : c.th, c.tb, c.bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, mp.act))
+        return RMSMP_ERR_CUDA;
     // packed weight regions: rows of Kp/2 (4-bit) and Kp (8-bit) bytes, boxes of 16 rows x one k-block
     auto make_w = [&](CUtensorMap* m, const uint8_t* base, int rows, int pitch, int box_bytes) -> bool {
         if (rows <= 0) return true;

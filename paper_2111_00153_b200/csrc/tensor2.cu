@@ -56,7 +56,7 @@ struct PairCfg {
 };
 
 struct PairMaps {
-    CUtensorMap act, wexp, out_full, out_tail;
+    CUtensorMap act[4], wexp, out_full, out_tail;      // act: one map, or one per parity sub-grid (stride 2)
 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -249,7 +249,6 @@ pair_kernel(const Problem p, const PairCfg cfg, const __grid_constant__ PairMaps
             const int64_t nt = tile / cfg.nbt;
             const int blk = (int)(tile - nt * cfg.nbt) * 2 + (int)rank;        // this CTA's row block
             const HalfPos hp = half_pos(p, cfg, 2 * nt + rank);               // this CTA's half of the pixels
-            const int y_base = hp.h0 * p.stride - p.pad;
             int tap = 0, cc = 0, ti = 0, tj = 0;
             for (int kb = 0; kb < cfg.nkb; kb += kSub2, ++g) {
                 const int nsub = min(kSub2, cfg.nkb - kb);
@@ -264,7 +263,10 @@ pair_kernel(const Problem p, const PairCfg cfg, const __grid_constant__ PairMaps
                 const uint32_t fb = lead_full + 8 * s;
                 for (int u = 0; u < nsub; ++u) {
                     if (!skip) {
-                        if (is_b) pair_load_4d(sB + (s * kSub2 + u) * kStageB, &maps.act, fb, cc * 128, tj - p.pad, y_base + ti, hp.b0);
+                        if (is_b) {
+                            const TapBox tb = tap_box(p, hp.h0, ti, tj);
+                            pair_load_4d(sB + (s * kSub2 + u) * kStageB, &maps.act[tb.map], fb, cc * 128, tb.x, tb.y, hp.b0);
+                        }
                         else pair_load_2d(sA + (s * kSub2 + u) * kStageA, &maps.wexp, fb, tap * p.Cp + cc * 128, blk * kBlockRows);
                     }
                     if (++cc == cfg.cpt) { cc = 0; ++tap; if (++tj == p.kw) { tj = 0; ++ti; } }
@@ -481,16 +483,7 @@ rmsmp_status launch_pair(const Problem& p, cudaStream_t st)
     if (!enc) return RMSMP_ERR_CUDA;
     PairMaps mp;
     memset(&mp, 0, sizeof(mp));
-    {
-        const cuuint64_t gdim[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
-        const cuuint64_t gstr[3] = {(cuuint64_t)p.pix_pitch, (cuuint64_t)p.pix_pitch * p.W, (cuuint64_t)p.pix_pitch * p.W * p.H};
-        const cuuint32_t box[4] = {128u, (cuuint32_t)(p.Wo * p.stride), (cuuint32_t)(c.th * p.stride), (cuuint32_t)c.tb};
-        const cuuint32_t estr[4] = {1u, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1u};
-        if (enc(&mp.act, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(p.act), gdim, gstr, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return RMSMP_ERR_CUDA;
-    }
+    if (!encode_act_maps_4(p, 128, c.th, c.tb, mp.act)) return RMSMP_ERR_CUDA;
     {
         const cuuint64_t gd[2] = {(cuuint64_t)p.Kp, (cuuint64_t)p.M};
         const cuuint64_t gs[1] = {(cuuint64_t)p.Kp};

@@ -224,6 +224,14 @@ CONV_CASES = [
     (200, 64, 2, 1, 0, 2, 9, 9),      # 64-byte pixels, even tap count, two row blocks (weights through the ring)
     (96, 64, 3, 2, 1, 3, 7, 7),       # 64-byte pixels, several images per tile, stride 2
     (64, 48, 1, 1, 0, 2, 12, 12),     # 64-byte pixels, one tap
+    (48, 32, 3, 2, 0, 2, 9, 11),      # stride 2 without padding, odd sizes: the parity sub-grids differ in extent
+    (32, 64, 5, 2, 2, 2, 10, 7),      # stride 2, 5x5: taps two rows / columns outside the image
+    (24, 32, 2, 2, 0, 3, 8, 6),       # stride 2, even kernel
+    (40, 32, 3, 3, 1, 2, 10, 13),     # stride 3: element-strided boxes (no parity split)
+    (300, 128, 3, 2, 1, 2, 28, 28),   # stride 2, three row blocks, tiles of whole output rows
+    (48, 64, 3, 1, 1, 3, 16, 8),      # resident weights, width a multiple of 8: one activation stage per kernel column
+    (64, 32, 3, 1, 1, 2, 24, 24),     # the same with one 32-code step per tap, tiles of several output rows
+    (100, 64, 3, 1, 1, 2, 40, 56),    # the same, ragged last row block, non-square image
 ]
 
 
