@@ -367,6 +367,198 @@ __global__ void __launch_bounds__(256, 2) grouped_kernel(const uint8_t* __restri
     }
 }
 
+// One-token form, software-pipelined across work items.  The profile of the plain form above
+// shows warps waiting on their weight loads four cycles out of eight: an item's loads are issued,
+// waited for, consumed, and only then does the warp look at its next item.  Here a warp walks a
+// flat sequence of steps -- a step is one 128-bit load per lane from each of the item's rows
+// (8 rows of 4-bit codes or 4 rows of Fixed-8 codes: 128 bytes per lane, 4 KB per warp) -- and the
+// loads of step i+1, which may belong to the next item or even the next layer, are issued before
+// step i is expanded and multiplied, so every warp has weight bytes in flight all the time.
+struct StreamItem {
+    const Problem* p;
+    const uint8_t* base;       // first row of the item
+    uint32_t pitch;            // bytes per packed row
+    int kind, nrows, nchunks;
+    int row_m;                 // lane r: original index of row r
+    float row_c;               // lane r: scale of row r
+};
+
+__device__ __forceinline__ bool stream_item(const uint8_t* table, int64_t w, int& pi, int lane, StreamItem& it)
+{
+    const GroupedTable* hdr = reinterpret_cast<const GroupedTable*>(table);
+    if (w >= hdr->total) return false;
+    const int64_t* cum = reinterpret_cast<const int64_t*>(table + sizeof(GroupedTable));
+    const Problem* probs = reinterpret_cast<const Problem*>(table + hdr->prob_off);
+    while (w >= cum[pi + 1]) ++pi;
+    const Problem& p = probs[pi];
+    const int li = (int)(w - cum[pi]);                       // one token: an item index inside the layer
+    const int iP = (p.nP + 7) >> 3, iF = (p.nF4 + 7) >> 3;
+    int pr0, rows_left;
+    if (li < iP) { it.kind = kPoT4; pr0 = li * 8; rows_left = p.nP - pr0; }
+    else if (li < iP + iF) { it.kind = kFixed4; pr0 = p.nP + (li - iP) * 8; rows_left = p.nP + p.nF4 - pr0; }
+    else { it.kind = kFixed8; pr0 = p.nP + p.nF4 + (li - iP - iF) * 4; rows_left = p.M - pr0; }
+    const int cap = (it.kind == kFixed8) ? 4 : 8;
+    it.p = &p;
+    it.nrows = rows_left < cap ? rows_left : cap;
+    it.nchunks = p.Cp >> 5;
+    if (it.kind == kFixed8) { it.pitch = (uint32_t)p.Kp; it.base = p.q8 + (size_t)(pr0 - p.nP - p.nF4) * it.pitch; }
+    else { it.pitch = (uint32_t)p.Kp >> 1; it.base = p.q4 + (size_t)pr0 * it.pitch; }
+    it.row_m = 0;
+    it.row_c = 0.0f;
+    if (lane < it.nrows) {
+        it.row_m = __ldg(p.perm + pr0 + lane);
+        it.row_c = __fmul_rn(__ldg(p.wstep + it.row_m), p.act_step);
+    }
+    return true;
+}
+
+// raw[r] = chunk `ch` of row r (4-bit kinds); raw[2r], raw[2r+1] = its two halves (Fixed-8).
+__device__ __forceinline__ void stream_load(const StreamItem& it, int ch, uint4 (&raw)[8], uint4 (&act)[2])
+{
+    const bool live = ch < it.nchunks;
+    // the token's 32 activation codes of this chunk travel with the weights (a ragged last chunk is
+    // fetched bytewise at compute time instead)
+    act[0] = act[1] = make_uint4(0, 0, 0, 0);
+    if (live && (ch << 5) + 32 <= it.p->Cin) {
+        const uint4* ap = reinterpret_cast<const uint4*>(it.p->act + (ch << 5));
+        act[0] = __ldg(ap);
+        act[1] = __ldg(ap + 1);
+    }
+    if (it.kind == kFixed8) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int rr = r < it.nrows ? r : it.nrows - 1;  // rows past the item's end repeat its last one
+            const uint4* src = reinterpret_cast<const uint4*>(it.base + (size_t)rr * it.pitch + ((size_t)ch << 5));
+            raw[2 * r] = live ? __ldcs(src) : make_uint4(0, 0, 0, 0);
+            raw[2 * r + 1] = live ? __ldcs(src + 1) : make_uint4(0, 0, 0, 0);
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const int rr = r < it.nrows ? r : it.nrows - 1;
+            const uint4* src = reinterpret_cast<const uint4*>(it.base + (size_t)rr * it.pitch + ((size_t)ch << 4));
+            raw[r] = live ? __ldcs(src) : make_uint4(0, 0, 0, 0);
+        }
+    }
+}
+
+__device__ __forceinline__ void stream_compute(const StreamItem& it, int ch, const uint4 (&raw)[8], const uint4 (&act)[2],
+                                               int (&acc)[8])
+{
+    if (ch >= it.nchunks) return;
+    const Problem& p = *it.p;
+    const int kp = ch << 5;
+    uint32_t a[8] = {act[0].x, act[0].y, act[0].z, act[0].w, act[1].x, act[1].y, act[1].z, act[1].w};
+    if (kp + 32 > p.Cin) {
+        const int8_t* ap = p.act + kp;                       // token 0
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t v = 0;
+#pragma unroll
+            for (int bb = 0; bb < 4; ++bb)
+                if (kp + q * 4 + bb < p.Cin) v |= (uint32_t)(uint8_t)ap[q * 4 + bb] << (8 * bb);
+            a[q] = v;
+        }
+    }
+    if (it.kind == kPoT4) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const uint32_t c[4] = {raw[r].x, raw[r].y, raw[r].z, raw[r].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {                    // eight codes at a time: few registers live
+                uint32_t w0, w1;
+                expand_pot_word(c[q], w0, w1);
+                acc[r] = __dp4a((int)w1, (int)a[2 * q + 1], __dp4a((int)w0, (int)a[2 * q], acc[r]));
+            }
+        }
+    } else if (it.kind == kFixed4) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const uint32_t c[4] = {raw[r].x, raw[r].y, raw[r].z, raw[r].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {                    // byte b: code b in the high, code 16 + b in the low nibble
+                acc[r] = __dp4a((int)(c[q] & 0xF0F0F0F0u), (int)a[q], acc[r]);
+                acc[r] = __dp4a((int)((c[q] << 4) & 0xF0F0F0F0u), (int)a[4 + q], acc[r]);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint32_t c[8] = {raw[2 * r].x, raw[2 * r].y, raw[2 * r].z, raw[2 * r].w,
+                                   raw[2 * r + 1].x, raw[2 * r + 1].y, raw[2 * r + 1].z, raw[2 * r + 1].w};
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[r] = __dp4a((int)c[q], (int)a[q], acc[r]);
+        }
+    }
+}
+
+__device__ __forceinline__ void stream_finish(const StreamItem& it, int lane, int (&acc)[8])
+{
+    const Problem& p = *it.p;
+    int mine = 0;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        int v = __reduce_add_sync(0xffffffffu, acc[r]);
+        if (it.kind == kFixed4) v >>= 4;                     // the Fixed-4 codes were expanded as 16 * value
+        if (lane == r) mine = v;
+        acc[r] = 0;
+    }
+    if (lane < it.nrows) {
+        const int64_t o = p.out_mn ? (int64_t)it.row_m * p.ld_out : (int64_t)it.row_m;
+        p.out[o] = __fmul_rn(__int2float_rn(mine), it.row_c);
+        if (p.acc) p.acc[o] = mine;
+    }
+}
+
+__global__ void __launch_bounds__(256, 2) grouped_stream_kernel(const uint8_t* __restrict__ gtable, int use_smem)
+{
+    extern __shared__ __align__(16) uint8_t s_table[];
+    const uint8_t* table = gtable;
+    if (use_smem) {
+        const int n16 = reinterpret_cast<const GroupedTable*>(gtable)->bytes >> 4;
+        for (int i = threadIdx.x; i < n16; i += blockDim.x)
+            reinterpret_cast<uint4*>(s_table)[i] = __ldg(reinterpret_cast<const uint4*>(gtable) + i);
+        __syncthreads();
+        table = s_table;
+    }
+    const int lane = threadIdx.x & 31;
+    int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    StreamItem cur, nxt;
+    int pi = 0;
+    if (!stream_item(table, w, pi, lane, cur)) return;
+    int ch = lane;
+    uint4 rc[8], rn[8], ac[2], an[2];
+    int acc[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) acc[r] = 0;
+    stream_load(cur, ch, rc, ac);
+    for (;;) {
+        const bool same = (ch - lane + 32) < cur.nchunks;    // warp-uniform: the item has another step
+        bool more = true;
+        if (same) {
+            stream_load(cur, ch + 32, rn, an);
+        } else {
+            w += nwarps;
+            more = stream_item(table, w, pi, lane, nxt);
+            if (more) stream_load(nxt, lane, rn, an);
+        }
+        stream_compute(cur, ch, rc, ac, acc);
+        if (same) {
+            ch += 32;
+        } else {
+            stream_finish(cur, lane, acc);
+            if (!more) break;
+            cur = nxt;
+            ch = lane;
+        }
+#pragma unroll
+        for (int r = 0; r < 8; ++r) rc[r] = rn[r];
+        ac[0] = an[0];
+        ac[1] = an[1];
+    }
+}
+
 size_t grouped_table_bytes(int count)
 {
     size_t off = sizeof(GroupedTable) + sizeof(int64_t) * (size_t)(count + 1);
@@ -403,7 +595,7 @@ int grouped_fill_table(const Problem* probs, int count, uint8_t* h_table)
 cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t total, int nt, cudaStream_t st)
 {
     int64_t blocks = (total + 7) / 8;
-    if (blocks > 148 * 2 * 4) blocks = 148 * 2 * 4;
+    if (blocks > 148 * 2) blocks = 148 * 2;                  // one resident wave: two blocks of 128-register threads per SM
     if (blocks < 1) blocks = 1;
     const int use_smem = table_bytes <= (size_t)kGroupedSmemMax;
     const size_t smem = use_smem ? table_bytes : 0;
@@ -411,12 +603,12 @@ cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t t
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(grouped_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupedSmemMax);
+        cudaError_t e = cudaFuncSetAttribute(grouped_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupedSmemMax);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(grouped_kernel<kTok>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupedSmemMax);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
     }
-    if (nt == 1) grouped_kernel<1><<<(unsigned)blocks, 256, smem, st>>>(d_table, use_smem);
+    if (nt == 1) grouped_stream_kernel<<<(unsigned)blocks, 256, smem, st>>>(d_table, use_smem);
     else grouped_kernel<kTok><<<(unsigned)blocks, 256, smem, st>>>(d_table, use_smem);
     return cudaGetLastError();
 }
