@@ -484,7 +484,12 @@ def run_suite(args):
     VAR = (("tensor_smem", R.VARIANT_TENSOR), ("tensor_workspace", "ws"), ("workspace_requant", "rq"),
            ("simt_dp4a", R.VARIANT_SIMT), ("shift_add", R.VARIANT_SHIFTADD))
 
+    def want(tag):
+        return not args.suite_filter or args.suite_filter in tag
+
     def bench_shape(cfg, name, M, Cin, k, stride, pad, B, H, ratio=RATIO, pool=1, only=None, iters=20):
+        if not want(cfg):
+            return
         conv = k > 1 or H > 1
         inst = [prep(M, Cin, k, ratio, 17 * i + M, conv) for i in range(pool)]
         Ho = (H + 2 * pad - k) // stride + 1
@@ -537,6 +542,8 @@ def run_suite(args):
     # config 5 as the natural cold stream: the whole BERT-large stack (24 x six linears, ~158 MB of
     # packed weights, larger than L2) in ONE grouped launch; the table upload is part of the call.
     for N in (1, 8):
+        if not want("grouped"):
+            break
         keep, items, wbytes, ops, alg = [], [], 0, 0, 0
         for l in range(24):
             for (M, K) in ((1024, 1024),) * 4 + ((4096, 1024), (1024, 4096)):
@@ -582,6 +589,9 @@ def main():
                          "activation path; 1: everything on one stream")
     ap.add_argument("--suite", action="store_true",
                     help="side-by-side timing of the kernel variants on all five configurations (not the headline)")
+    ap.add_argument("--suite-filter", default=None,
+                    help="with --suite: only the rows whose configuration tag contains this text "
+                         "(config1 .. config5, or 'grouped' for the one-launch BERT-large stack)")
     ap.add_argument("--layers", default=None,
                     help="comma-separated layer names: run one instance of each (profiling runs)")
     args = ap.parse_args()

@@ -64,10 +64,6 @@ struct TensorCfg {
     int nA, nB, nR;        // ring depths: expanded weights, activations, raw weights
     uint32_t raw_bytes;    // one raw stage
     int out_bufs;          // staging buffers per epilogue warp (1 or 2)
-    int fastcvt;           // 1: every |accumulator| of this problem is below 2^22, so int -> float is done exactly with
-                           //    an integer add and a float subtract (see acc_to_float_small) instead of a conversion
-                           //    instruction, whose pipe runs at a fraction of the arithmetic rate and bounds the
-                           //    epilogue of output-bound layers
     int pre;               // 1: the A operand comes expanded (int8) from a workspace, no expander work
     int dup;               // 1 (pre mode, M <= 64): rows 0..63 are loaded twice, into lanes 0..63 and 64..127, so that all
                            //    four tensor-memory quarters hold valid rows and every epilogue warp has work
@@ -233,14 +229,6 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32])
                    "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
                    "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
                  :: "memory");
-}
-
-// Exact float value of an integer |a| < 2^22 without a conversion instruction: the bit pattern of
-// 1.5 * 2^23 plus a is the float 12582912 + a (floats in [2^23, 2^24) are the integers), and
-// subtracting 12582912 back is exact.
-__device__ __forceinline__ float acc_to_float_small(int a)
-{
-    return __fsub_rn(__int_as_float(a + 0x4B400000), 12582912.0f);
 }
 
 // ------------------------------------------------------------------ per-tile row bookkeeping
@@ -825,19 +813,11 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                         if (!p.out_mn) {
                             // [pixel][row]: the warp writes 128 contiguous bytes per pixel
                             const uint32_t a0 = stg + lane * 4;
-                            if (cfg.fastcvt && !sub) {
 #pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    const uint32_t w = __float_as_uint(__fmul_rn(acc_to_float_small((int)v[j] >> shift), scale));
-                                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 128), "r"(w) : "memory");
-                                }
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    const int a = (int)v[j] >> shift;
-                                    const uint32_t w = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
-                                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 128), "r"(w) : "memory");
-                                }
+                            for (int j = 0; j < 32; ++j) {
+                                const int a = (int)v[j] >> shift;
+                                const uint32_t w = sub ? (uint32_t)a : __float_as_uint(__fmul_rn(__int2float_rn(a), scale));
+                                asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + j * 128), "r"(w) : "memory");
                             }
                         } else {
                             // [row][pixel], 16-byte chunks swizzled by row (matches the 128-byte-swizzled store map)
@@ -1032,9 +1012,6 @@ bool plan(const Problem& p, TensorCfg& c)
     c.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.n_mma >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
     c.tail_rows = c.npix & 31;
     c.tma_store = 0;
-    // |acc| <= K * 127 * 15 (4-bit activation codes, 8-bit weights at most), times 16 while Fixed-4 rows are
-    // expanded as 16 * value in shared-memory expansion mode
-    c.fastcvt = ((int64_t)p.kh * p.kw * p.Cin * 127 * 15 * (p.wexp ? 1 : 16) < (1ll << 22)) ? 1 : 0;
     c.dup = 0;
     c.ares = 0;
     c.epi_warps = kNumEpiWarps;
