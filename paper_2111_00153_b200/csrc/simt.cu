@@ -218,7 +218,7 @@ constexpr int kGroupedSmemMax = 96 * 1024;
 __host__ __device__ inline int grouped_rw(int kind, int nt)
 {
     if (nt == 1) return kind == kFixed8 ? 4 : 8;
-    return 2;
+    return kind == kFixed8 ? 2 : 4;
 }
 
 template <int KIND>
@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(256, 2) grouped_kernel(const uint8_t* __restri
     const GroupedTable* hdr = reinterpret_cast<const GroupedTable*>(table);
     const int64_t* cum = reinterpret_cast<const int64_t*>(table + sizeof(GroupedTable));
     const Problem* probs = reinterpret_cast<const Problem*>(table + hdr->prob_off);
-    constexpr int RW4 = (NT == 1) ? 8 : 2, RW8 = (NT == 1) ? 4 : 2;
+    constexpr int RW4 = (NT == 1) ? 8 : 4, RW8 = (NT == 1) ? 4 : 2;
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -352,8 +352,16 @@ __global__ void __launch_bounds__(256, 2) grouped_kernel(const uint8_t* __restri
         const int64_t local = w - cum[pi];
         const int iP = (p.nP + RW4 - 1) / RW4, iF = (p.nF4 + RW4 - 1) / RW4, i8 = (p.n8 + RW8 - 1) / RW8;
         const int ipg = iP + iF + i8;
-        const int li = (int)(local % ipg);
-        const int64_t n0 = (local / ipg) * NT;
+        int li;
+        int64_t n0;
+        if ((local >> 32) == 0) {                            // the usual case: 32-bit division
+            const uint32_t q = (uint32_t)local / (uint32_t)ipg;
+            li = (int)((uint32_t)local - q * (uint32_t)ipg);
+            n0 = (int64_t)q * NT;
+        } else {
+            li = (int)(local % ipg);
+            n0 = (local / ipg) * NT;
+        }
         if (li < iP) {
             const int r0 = li * RW4;
             grouped_rows<kPoT4, NT, RW4>(p, r0, min(RW4, p.nP - r0), n0, lane);
