@@ -295,10 +295,15 @@ __device__ __forceinline__ void expand_task(uint32_t meta, uint32_t raw_stage, u
 
 // kM2: a tile covers two row blocks (TensorCfg::m2), compiled separately so that the common form keeps its registers.
 // kRQ: the epilogue writes the next layer's activation codes instead of fp32 (Problem::rq_codes).
-template <int kM2, int kRQ>
+// kMode: which of the kernel's forms this instantiation is (the host picks it from the plan): 0 codes expanded in
+//        shared memory; 1 expanded weights from a workspace through the ring; 2 the same, weights resident in
+//        shared memory; 3 resident weights and three taps per activation stage.  A compile-time constant so that
+//        an instantiation carries only the code of its own form.
+template <int kM2, int kRQ, int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
 tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps maps)
 {
+    constexpr bool kPre = kMode != 0, kAres = kMode >= 2, kTps3 = kMode == 3;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sA = smem_base;
@@ -318,7 +323,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxRing; ++s) {
-            mbar_init(bar_fullA + 8 * s, cfg.pre ? 1 : 4);   // producer (+ bytes), or the four warps of one expander group
+            mbar_init(bar_fullA + 8 * s, kPre ? 1 : 4);   // producer (+ bytes), or the four warps of one expander group
             mbar_init(bar_emptyA + 8 * s, 1);    // tcgen05.commit
             mbar_init(bar_fullB + 8 * s, 1);     // producer (+ transaction bytes)
             mbar_init(bar_emptyB + 8 * s, 1);    // tcgen05.commit
@@ -347,11 +352,11 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
 
     // Workspace mode splits the producer: one thread can start a bulk tensor copy only every few
     // hundred cycles, so the activation boxes and the weight boxes are issued by two different warps.
-    const bool pre_b_producer = cfg.pre && warp == 0;
-    const bool pre_a_producer = cfg.pre && !cfg.ares && warp == 2;
+    const bool pre_b_producer = kPre && warp == 0;
+    const bool pre_a_producer = kPre && !kAres && warp == 2;
     if (pre_b_producer || pre_a_producer) {
         if (lane == 0) {
-            if (pre_b_producer && cfg.ares && my_tiles > 0) {
+            if (pre_b_producer && kAres && my_tiles > 0) {
                 // resident weights: every k-block's rows, once
                 mbar_arrive_expect_tx(bar_fullA, (uint32_t)(cfg.nkb * cfg.a_bytes));
                 int tap = 0, cc = 0;
@@ -383,7 +388,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 int tap = 0, cc = 0, ti = 0, tj = 0;
                 for (int kb = 0; kb < cfg.nkb; ++kb) {
                     if (!mbar_wait(bar_e + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
-                    if (pre_b_producer && cfg.tps > 1) {
+                    if (pre_b_producer && kTps3) {
                         if (cfg.colshift) {
                             // one stage = one column shift: the th + kh - 1 input rows the tile needs, fetched once
                             // and read by the kh taps of that column at row offsets (see TensorCfg::colshift)
@@ -427,7 +432,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         {
             uint32_t sb = 0, phB = 0, sr = 0, phR = 0;
             bool ok = true;
-            if (cfg.ares && lane == 0 && my_tiles > 0) {
+            if (kAres && lane == 0 && my_tiles > 0) {
                 // resident weights: every k-block's rows, once
                 mbar_arrive_expect_tx(bar_fullA, (uint32_t)(cfg.nkb * cfg.a_bytes));
                 int tap = 0, cc = 0;
@@ -466,9 +471,9 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 int tap = 0, cc = 0;
                 for (int kb = 0; kb < cfg.nkb; ++kb) {
                     const int c0 = cc * cfg.bk, koff = tap * p.Cp + c0;
-                    if (cfg.ares) {
+                    if (kAres) {
                         // weights are resident
-                    } else if (cfg.pre) {
+                    } else if (kPre) {
                         // weights already expanded: one swizzled 128-row box straight into the A stage
                         if (!mbar_wait_warp(bar_emptyA + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
                         if (lane == 0) {
@@ -516,7 +521,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
             uint32_t sa = 0, phA = 0, sb = 0, phB = 0, it = 0;
             const uint64_t desc_a0 = smem_desc_kmajor(sA, cfg.bk), desc_b0 = smem_desc_kmajor(sB, cfg.bk);
             const uint32_t desc_lo0_a = (uint32_t)desc_a0, desc_lo0_b = (uint32_t)desc_b0, desc_hi = (uint32_t)(desc_a0 >> 32);
-            bool have_a = !cfg.ares || my_tiles == 0 || mbar_wait(bar_fullA, 0, abort_flag);
+            bool have_a = !kAres || my_tiles == 0 || mbar_wait(bar_fullA, 0, abort_flag);
             for (int64_t tile = first; tile < cfg.ntiles && have_a && !*abort_flag; tile += step, ++it) {
                 // one accumulator per tile, alternating; or (two row blocks per tile) both, every tile
                 const uint32_t ab = kM2 ? 0u : (it & 1);
@@ -526,7 +531,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 const uint32_t d_tmem = tmem_base + ab * kTileN;
                 bool ok = true;
                 int cc = 0;
-                if (cfg.tps > 1) {
+                if (kTps3) {
                     // resident weights, three 64-byte k-blocks per activation stage (never with two row blocks):
                     // the taps of a kernel row in three sub-buffers, or (colshift) the taps of a kernel COLUMN
                     // reading one buffer at three row offsets
@@ -552,7 +557,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                         b_lo += b_step;
                         if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; b_lo = desc_lo0_b; }
                     }
-                } else if (!cfg.ares && cfg.bk == 128 && cfg.last_ksteps == 4) {
+                } else if (!kAres && cfg.bk == 128 && cfg.last_ksteps == 4) {
                     // The common deep-K form, kept as short as it gets: every k-block is four MMAs (eight
                     // with two row blocks) on a full 128-byte stage of each ring.
                     const uint32_t a_step = (uint32_t)cfg.a_bytes >> 4, b_step = (uint32_t)cfg.b_bytes >> 4;
@@ -589,11 +594,11 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 } else {
                     const bool uniform = (cfg.last_ksteps == (cfg.bk >> 5));      // every k-block has the same depth
                     const uint32_t a_step = (uint32_t)cfg.a_bytes >> 4, b_step = (uint32_t)cfg.b_bytes >> 4;
-                    uint32_t a_lo = cfg.ares ? desc_lo0_a : desc_lo0_a + sa * a_step;
+                    uint32_t a_lo = kAres ? desc_lo0_a : desc_lo0_a + sa * a_step;
                     uint32_t b_lo = desc_lo0_b + sb * b_step;
                     for (int kb = 0; kb < cfg.nkb; ++kb) {
                         if (!mbar_wait(bar_fullB + 8 * sb, phB, abort_flag) ||
-                            (!cfg.ares && !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag))) { ok = false; break; }
+                            (!kAres && !mbar_wait(bar_fullA + 8 * sa, phA, abort_flag))) { ok = false; break; }
                         tc_fence_after();
                         const int ksteps = (uniform || cc != cfg.cpt - 1) ? (cfg.bk >> 5) : cfg.last_ksteps;
                         if (issuer) mma_i8_halves(d_tmem, a_lo, b_lo, desc_hi, cfg.idesc, kb ? 1u : 0u);
@@ -610,11 +615,11 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                             for (int ks = 1; ks < ksteps; ++ks)
                                 if (issuer) mma_i8_halves(d_tmem + kTileN, a1 + 2 * ks, b_lo + 2 * ks, desc_hi, cfg.idesc, 1u);
                         }
-                        if (!cfg.ares && issuer) mma_commit(bar_emptyA + 8 * sa);
+                        if (!kAres && issuer) mma_commit(bar_emptyA + 8 * sa);
                         if (issuer) mma_commit(bar_emptyB + 8 * sb);
                         a_lo += a_step;
                         b_lo += b_step;
-                        if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; if (!cfg.ares) a_lo = desc_lo0_a; }
+                        if (++sa == (uint32_t)cfg.nA) { sa = 0; phA ^= 1; if (!kAres) a_lo = desc_lo0_a; }
                         if (++sb == (uint32_t)cfg.nB) { sb = 0; phB ^= 1; b_lo = desc_lo0_b; }
                         if (!uniform && ++cc == cfg.cpt) cc = 0;
                     }
@@ -624,7 +629,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 if (kM2 && issuer) mma_commit(bar_tfull + 8);
             }
         }
-    } else if (!cfg.pre && warp < 2 + kNumExpWarps) {
+    } else if (!kPre && warp < 2 + kNumExpWarps) {
         // ---------------------------------------------------------- expanders
         const int grp = (warp - 2) >> 2;                 // which k-blocks: g % kGroups == grp
         const int et = ((warp - 2) & 3) * 32 + lane;     // 0..127 inside the group
@@ -632,7 +637,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         const int slot0 = et >> 2;                       // rows slot0 + 32*i of the tile's sorted order
         // tile look-ahead: one tile, or kGroups tiles when every tile is a single k-block
         const int64_t look = (cfg.nkb == 1) ? kGroups : 1;
-        const int64_t total = cfg.pre ? 0 : my_tiles * cfg.nkb;   // nothing to expand in pre mode
+        const int64_t total = kPre ? 0 : my_tiles * cfg.nkb;   // nothing to expand in pre mode
         int64_t g = grp;                                 // this CTA's k-block counter
         int64_t tl = g / cfg.nkb;                        // local tile index of g
         int kb = (int)(g - tl * cfg.nkb);
@@ -643,8 +648,8 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
         auto tile_of = [&](int64_t local) -> int64_t { return local < my_tiles ? first + local * step : -1; };
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            cur[i] = cfg.pre ? 0u : make_meta(p, tile_of(tl), slot0 + 32 * i, q);
-            nxt[i] = cfg.pre ? 0u : make_meta(p, tile_of(tl + look), slot0 + 32 * i, q);
+            cur[i] = kPre ? 0u : make_meta(p, tile_of(tl), slot0 + 32 * i, q);
+            nxt[i] = kPre ? 0u : make_meta(p, tile_of(tl + look), slot0 + 32 * i, q);
         }
         while (g < total) {
             const int ksteps = (cc == cfg.cpt - 1) ? cfg.last_ksteps : 4;
@@ -730,7 +735,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 shift = 0;
                 if (row_ok) {
                     scale = __fmul_rn(__ldg(p.wstep + m), p.act_step);
-                    shift = (!cfg.pre && __ldg(p.kind + m) == kFixed4) ? 4 : 0;   // expanders store Fixed-4 codes as 16 * value
+                    shift = (!kPre && __ldg(p.kind + m) == kFixed4) ? 4 : 0;   // expanders store Fixed-4 codes as 16 * value
                 }
             }
             if (!mbar_wait_warp(bar_tfull + 8 * ab, tpar, abort_flag)) { alive = false; break; }
@@ -1170,25 +1175,28 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
         c.tma_store = ok ? 1 : 0;
     }
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(tensor_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
-            cudaFuncSetAttribute(tensor_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
-            cudaFuncSetAttribute(tensor_kernel<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
-            cudaFuncSetAttribute(tensor_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
+    // the kernel's form (see tensor_kernel): [mode][two row blocks][re-quantizing epilogue]
+    typedef void (*KernelFn)(const Problem, const TensorCfg, const Maps);
+    static const KernelFn table[4][2][2] = {
+        {{tensor_kernel<0, 0, 0>, nullptr}, {nullptr, nullptr}},
+        {{tensor_kernel<0, 0, 1>, tensor_kernel<0, 1, 1>}, {tensor_kernel<1, 0, 1>, tensor_kernel<1, 1, 1>}},
+        {{tensor_kernel<0, 0, 2>, tensor_kernel<0, 1, 2>}, {nullptr, nullptr}},
+        {{tensor_kernel<0, 0, 3>, tensor_kernel<0, 1, 3>}, {nullptr, nullptr}},
+    };
+    const int mode = !c.pre ? 0 : (!c.ares ? 1 : (c.tps > 1 ? 3 : 2));
+    const int i2 = c.m2 ? 1 : 0, irq = p.rq_codes ? 1 : 0;
+    const KernelFn fn = table[mode][i2][irq];
+    if (!fn) return RMSMP_ERR_VARIANT;
+    static bool attr_set[4][2][2] = {};
+    if (!attr_set[mode][i2][irq]) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
             cudaGetLastError();
             return RMSMP_ERR_CUDA;
         }
-        attr_set = true;
+        attr_set[mode][i2][irq] = true;
     }
     const int grid = (int)std::min<int64_t>(c.ntiles, sm_count());
-    if (p.rq_codes) {
-        if (c.m2) tensor_kernel<1, 1><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
-        else tensor_kernel<0, 1><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
-    } else {
-        if (c.m2) tensor_kernel<1, 0><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
-        else tensor_kernel<0, 0><<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
-    }
+    fn<<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
     if (cudaGetLastError() != cudaSuccess) return RMSMP_ERR_CUDA;
     return RMSMP_OK;
 }
