@@ -299,11 +299,16 @@ __device__ __forceinline__ void expand_task(uint32_t meta, uint32_t raw_stage, u
 //        shared memory; 1 expanded weights from a workspace through the ring; 2 the same, weights resident in
 //        shared memory; 3 resident weights and three taps per activation stage.  A compile-time constant so that
 //        an instantiation carries only the code of its own form.
-template <int kM2, int kRQ, int kMode>
+// kOut:  1 when the output is fp32 [N][M] through bulk stores without an accumulator dump (the common case): the
+//        epilogue then carries only that path; 0 decides at run time.
+template <int kM2, int kRQ, int kMode, int kOut>
 __global__ void __launch_bounds__(kThreads, 1)
 tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps maps)
 {
     constexpr bool kPre = kMode != 0, kAres = kMode >= 2, kTps3 = kMode == 3;
+    const bool use_tma_store = kOut ? true : (cfg.tma_store != 0);
+    const bool out_mn = kOut ? false : (p.out_mn != 0);
+    int32_t* const acc_out = kOut ? nullptr : p.acc;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sA = smem_base;
@@ -758,7 +763,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                 if (kRQ) {
                     // y as in the fp32 epilogue, then the activation quantizer's arithmetic on it;
                     // one code byte per output, 32 pixels x 32 rows = 1 KB per chunk
-                    if (cfg.tma_store) {
+                    if (use_tma_store) {
                         const bool tail = cfg.tail_rows && (c == (cfg.npix >> 5));
                         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                         __syncwarp();
@@ -804,9 +809,9 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                             }
                         }
                     }
-                } else if (cfg.tma_store) {
+                } else if (use_tma_store) {
                     const bool tail = cfg.tail_rows && (c == (cfg.npix >> 5));
-                    const int nsub = p.acc ? 2 : 1;
+                    const int nsub = acc_out ? 2 : 1;
                     for (int sub = 0; sub < nsub; ++sub) {
                         const uint32_t stg = my_stage + (cfg.out_bufs == 2 ? (stg_count & 1) * kWarpStage : 0);
                         ++stg_count;
@@ -815,7 +820,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                             else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                         }
                         __syncwarp();                    // the buffer's previous store has been read out
-                        if (!p.out_mn) {
+                        if (!out_mn) {
                             // [pixel][row]: the warp writes 128 contiguous bytes per pixel
                             const uint32_t a0 = stg + lane * 4;
 #pragma unroll
@@ -845,14 +850,14 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                             const CUtensorMap* map = sub ? (tail ? &maps.acc_tail : &maps.acc_full)
                                                          : (tail ? &maps.out_tail : &maps.out_full);
                             const int cm = blk * kBlockRows + row0, cn = (int)(n0 + c * 32);
-                            if (!p.out_mn) tma_store_2d(map, stg, cm, cn); else tma_store_2d(map, stg, cn, cm);
+                            if (!out_mn) tma_store_2d(map, stg, cm, cn); else tma_store_2d(map, stg, cn, cm);
                         }
                     }
                 } else if (row_ok) {
                     // direct stores: outputs whose leading dimension or base rules out bulk stores
-                    if (!p.out_mn) {
+                    if (!out_mn) {
                         float* o = p.out + (n0 + c * 32) * p.ld_out + m;
-                        int32_t* oa = p.acc ? p.acc + (n0 + c * 32) * p.ld_out + m : nullptr;
+                        int32_t* oa = acc_out ? acc_out + (n0 + c * 32) * p.ld_out + m : nullptr;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             if (j < jmax) {
@@ -863,7 +868,7 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
                         }
                     } else {
                         float* o = p.out + (int64_t)m * p.ld_out + n0 + c * 32;
-                        int32_t* oa = p.acc ? p.acc + (int64_t)m * p.ld_out + n0 + c * 32 : nullptr;
+                        int32_t* oa = acc_out ? acc_out + (int64_t)m * p.ld_out + n0 + c * 32 : nullptr;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             if (j < jmax) {
@@ -1175,25 +1180,27 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
         c.tma_store = ok ? 1 : 0;
     }
 
-    // the kernel's form (see tensor_kernel): [mode][two row blocks][re-quantizing epilogue]
+    // the kernel's form (see tensor_kernel): [mode][two row blocks][1: re-quantizing epilogue, 2: plain fp32 [N][M] bulk-store output]
     typedef void (*KernelFn)(const Problem, const TensorCfg, const Maps);
-    static const KernelFn table[4][2][2] = {
-        {{tensor_kernel<0, 0, 0>, nullptr}, {nullptr, nullptr}},
-        {{tensor_kernel<0, 0, 1>, tensor_kernel<0, 1, 1>}, {tensor_kernel<1, 0, 1>, tensor_kernel<1, 1, 1>}},
-        {{tensor_kernel<0, 0, 2>, tensor_kernel<0, 1, 2>}, {nullptr, nullptr}},
-        {{tensor_kernel<0, 0, 3>, tensor_kernel<0, 1, 3>}, {nullptr, nullptr}},
+    static const KernelFn table[4][2][3] = {
+        {{tensor_kernel<0, 0, 0, 0>, nullptr, tensor_kernel<0, 0, 0, 1>}, {nullptr, nullptr, nullptr}},
+        {{tensor_kernel<0, 0, 1, 0>, tensor_kernel<0, 1, 1, 0>, tensor_kernel<0, 0, 1, 1>},
+         {tensor_kernel<1, 0, 1, 0>, tensor_kernel<1, 1, 1, 0>, tensor_kernel<1, 0, 1, 1>}},
+        {{tensor_kernel<0, 0, 2, 0>, tensor_kernel<0, 1, 2, 0>, tensor_kernel<0, 0, 2, 1>}, {nullptr, nullptr, nullptr}},
+        {{tensor_kernel<0, 0, 3, 0>, tensor_kernel<0, 1, 3, 0>, tensor_kernel<0, 0, 3, 1>}, {nullptr, nullptr, nullptr}},
     };
     const int mode = !c.pre ? 0 : (!c.ares ? 1 : (c.tps > 1 ? 3 : 2));
-    const int i2 = c.m2 ? 1 : 0, irq = p.rq_codes ? 1 : 0;
-    const KernelFn fn = table[mode][i2][irq];
+    const int i2 = c.m2 ? 1 : 0;
+    const int io = p.rq_codes ? 1 : ((c.tma_store && !p.out_mn && !p.acc) ? 2 : 0);
+    const KernelFn fn = table[mode][i2][io];
     if (!fn) return RMSMP_ERR_VARIANT;
-    static bool attr_set[4][2][2] = {};
-    if (!attr_set[mode][i2][irq]) {
+    static bool attr_set[4][2][3] = {};
+    if (!attr_set[mode][i2][io]) {
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
             cudaGetLastError();
             return RMSMP_ERR_CUDA;
         }
-        attr_set[mode][i2][irq] = true;
+        attr_set[mode][i2][io] = true;
     }
     const int grid = (int)std::min<int64_t>(c.ntiles, sm_count());
     fn<<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
