@@ -367,7 +367,7 @@ def run_ours(args):
 # dram bytes (read + write) of the 19 convolution launches of one step at batch 256, from an ncu
 # capture of this kernel (profiles/bench_resnet18_stack_launch_list.md); reported only for that
 # configuration.  Set back to None whenever tensor_kernel changes.
-TRAFFIC_PER_STEP_BYTES = 1257.6e6
+TRAFFIC_PER_STEP_BYTES = 1256.0e6
 
 
 def load_peaks():
