@@ -152,7 +152,8 @@ def test_config4_resnet18_layer_batch4_full(L):
 
 
 BIG = [L for L in synth.resnet18_convs() if L.name in
-       ("l1.conv3x3", "l2.conv3x3_s2", "l2.down1x1_s2", "l3.conv3x3", "l4.conv3x3")]
+       ("l1.conv3x3", "l2.conv3x3_s2", "l2.conv3x3", "l2.down1x1_s2", "l3.conv3x3_s2", "l3.conv3x3",
+        "l4.conv3x3_s2", "l4.conv3x3", "l4.down1x1_s2")]   # every kernel form the benchmark's stack runs on
 
 
 @pytest.mark.parametrize("L", BIG, ids=lambda L: L.name)
