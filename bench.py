@@ -334,6 +334,13 @@ def run_ours(args):
         return
 
     peaks, peak_src = load_peaks()
+    # tensor-bound part of the stack (the long-K layers that run on the two-CTA kernel) against the INT8
+    # tensor-core rate measured in this run by the library's MMA-only loop (operands resident in shared memory)
+    status_word = torch.zeros(4, dtype=torch.int32, device="cuda")
+    i8_peak, _ = R.rmsmp_measure_mma_peak(status_word, False, 256, 20000)
+    tb = [(layer_ops(h["L"], batch), float(ms)) for h, ms in zip(H, conv_ms_layer)
+          if h["L"].K >= 2048 and h["L"].M % 256 == 0]
+    tensor_tops = (sum(o for o, _ in tb) / (sum(m for _, m in tb) * 1e-3) / 1e12) if tb else None
     out = {
         "metric": METRIC, "value": whole_job_tops(ops_step, world, ms_step), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
@@ -353,6 +360,11 @@ def run_ours(args):
                      "traffic": TRAFFIC_PER_STEP_BYTES if (batch == BATCH and use_ws and not args.layers) else None,
                      "algorithmic_bytes_per_step": float(alg.sum()), "kernel_ms_per_step": conv_total_ms,
                      "kernel_tops": ops_step / (conv_total_ms * 1e-3) / 1e12},
+        "roofline_tensor": ({"bound": "tensor", "kernel": "pair_kernel (layers with K >= 2048 and M a multiple of 256)",
+                             "achieved": tensor_tops, "peak": i8_peak, "unit": "TOP/s", "frac": tensor_tops / i8_peak,
+                             "peak_source": "tcgen05.mma kind::i8 M=128 N=256 loop measured in this run (rmsmp_measure_mma_peak); "
+                                            "2 x measured bf16 GEMM = %.0f" % (2 * peaks["bf16_tflops"]),
+                             "layers": len(tb)} if tb and i8_peak > 0 else None),
         "per_layer": [{"name": h["L"].name, "M": h["L"].M, "K": h["L"].K, "N": d["N"], "ms": float(ms),
                        "tops": layer_ops(h["L"], batch) / (ms * 1e-3) / 1e12, "gbs": float(a / (ms * 1e-3) / 1e9)}
                       for h, d, ms, a in zip(H, D, conv_ms_layer, alg)],
