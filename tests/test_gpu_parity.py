@@ -232,6 +232,10 @@ CONV_CASES = [
     (48, 64, 3, 1, 1, 3, 16, 8),      # resident weights, width a multiple of 8: one activation stage per kernel column
     (64, 32, 3, 1, 1, 2, 24, 24),     # the same with one 32-code step per tap, tiles of several output rows
     (100, 64, 3, 1, 1, 2, 40, 56),    # the same, ragged last row block, non-square image
+    (64, 16, 7, 2, 3, 2, 32, 32),     # first-layer shape: 7x7 stride 2 pad 3 (3 input channels stored as 16, the rest zero)
+    (256, 64, 1, 1, 0, 2, 14, 14),    # bottleneck 1x1 expansions and reductions (ResNet-50 style)
+    (64, 256, 1, 1, 0, 2, 14, 14),
+    (32, 32, 3, 1, 1, 2, 16, 16),     # depthwise-separable networks' pointwise/3x3 sizes with few channels
 ]
 
 

@@ -186,6 +186,22 @@ def test_config4_resnet18_layer_batch256_sampled(L):
     assert not np.isnan(y).any()                         # every output was written
 
 
+def test_resnet18_first_layer_7x7_batch4_full():
+    """The 7x7 stride-2 first convolution at ImageNet size, its 3 input channels stored as 16 (zeros
+    beyond the third) so that a pixel is one 16-byte granule: every output against the oracle."""
+    M, Cin, k, B, H = 64, 16, 7, 4, 224
+    g = synth.rng(4, 777)
+    W = synth.weights_kaiming(g, M, Cin, k, k)
+    W[:, 3:] = 0.0
+    x = synth.act_halfnormal(g, (B, H, H, Cin))
+    x[..., 3:] = 0.0
+    scheme, bits = R.rmsmp_assign_rows(W, synth.RATIO_RMSMP1)
+    alpha = synth.alpha_rows(W)
+    codes, step, y = _run_conv_device(W, scheme, bits, alpha, x, 2, 3, R.ACT_U4)
+    _, ws, acc, y_ref = O.layer_conv(W, scheme, bits, alpha, codes, step, 2, 3)
+    assert np.array_equal(y.view(np.uint32), y_ref.reshape(-1, M).view(np.uint32))
+
+
 # ------------------------------------------------------------------ config 5: weight-bound small-N sweep
 
 @pytest.mark.parametrize("ratio", synth.RATIO_SWEEP, ids=lambda r: "%d-%d-%d" % r)
