@@ -200,7 +200,11 @@ def run_ours(args):
     # latency-bound launches) does not depend on its activations, so it runs on a side stream and
     # overlaps the activation quantizer / the previous layer's tail.  The convolution waits for
     # both; the next step's pack of a layer waits for this step's convolution of it (same buffers).
-    side = torch.cuda.Stream() if args.streams == 2 else None
+    side = torch.cuda.Stream() if args.streams >= 2 else None
+    # --streams 3 (not the default: the convolution's own duration is then no longer measured in isolation):
+    # the activation quantizer of layer i+1 also leaves the main stream and runs beside the convolution of layer i
+    qs = torch.cuda.Stream() if args.streams == 3 else None
+    qdone = [torch.cuda.Event() for _ in layers]
     ready = [torch.cuda.Event() for _ in layers]
     done = [torch.cuda.Event() for _ in layers]
     first_use = [True]
@@ -219,7 +223,16 @@ def run_ours(args):
                 R.rmsmp_expand_weights(h["lay"], d["packed"], d["ws"], stream=ws_stream)
             if side is not None:
                 ready[i].record(side)
-            st = R.rmsmp_quantize_act(d["x"], d["x"].numel(), synth.ALPHA_ACT, R.ACT_U4, d["codes"], stream=stream)
+            if qs is not None:
+                if first_use[0]:
+                    qs.wait_stream(stream)
+                else:
+                    qs.wait_event(done[i])                   # the previous step's convolution has read these codes
+                st = R.rmsmp_quantize_act(d["x"], d["x"].numel(), synth.ALPHA_ACT, R.ACT_U4, d["codes"], stream=qs)
+                qdone[i].record(qs)
+                stream.wait_event(qdone[i])
+            else:
+                st = R.rmsmp_quantize_act(d["x"], d["x"].numel(), synth.ALPHA_ACT, R.ACT_U4, d["codes"], stream=stream)
             if side is not None:
                 stream.wait_event(ready[i])
             if ev is not None:
@@ -596,9 +609,10 @@ def main():
     ap.add_argument("--variant", default="workspace", choices=["workspace", "smem"],
                     help="tensor-core path: expand the weight codes once into scratch memory (default) "
                          "or in shared memory per tile")
-    ap.add_argument("--streams", type=int, default=2, choices=[1, 2],
+    ap.add_argument("--streams", type=int, default=2, choices=[1, 2, 3],
                     help="2: each layer's weight path (pack, expand) runs on a side stream and overlaps the "
-                         "activation path; 1: everything on one stream")
+                         "activation path; 1: everything on one stream; 3: the activation quantizer too on a stream "
+                         "of its own, beside the previous layer's convolution (kernel timings then overlap)")
     ap.add_argument("--suite", action="store_true",
                     help="side-by-side timing of the kernel variants on all five configurations (not the headline)")
     ap.add_argument("--suite-filter", default=None,
