@@ -54,9 +54,10 @@ def layer_list():
 
 
 def host_layer(idx, L, batch, rank=0):
-    g = synth.rng(4, idx + 100 * rank)
-    W = synth.weights_kaiming(g, L.M, L.Cin, L.k, L.k)
-    x = synth.act_halfnormal(g, (batch, L.H, L.H, L.Cin))
+    """Weights are seeded by layer only (every rank holds the same, replicated model); the input
+    batch is seeded by layer and rank (every rank works on its own images)."""
+    W = synth.weights_kaiming(synth.rng(4, idx), L.M, L.Cin, L.k, L.k)
+    x = synth.act_halfnormal(synth.rng(4, 5000 + idx + 100 * rank), (batch, L.H, L.H, L.Cin))
     return W, x
 
 
@@ -93,6 +94,21 @@ def whole_job_tops(ops_per_gpu_step: int, world: int, ms_step: float) -> float:
     return world * ops_per_gpu_step / (ms_step * 1e-3) / 1e12
 
 
+def launch_ranks(argv, gpus: int) -> int:
+    """`bench.py --gpus N` started by hand (no WORLD_SIZE in the environment): start N ranks of this
+    same command, one per GPU, under torch.distributed.run on the loop-back address, and return
+    their exit code.  Rank 0 prints the one JSON line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--standalone", "--local-addr", "127.0.0.1",
+           "--nnodes=1", "--nproc-per-node", str(gpus), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def rank_env():
+    """(world, rank, local_rank) from the launcher's environment; (1, 0, 0) when there is none."""
+    return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
 # ---------------------------------------------------------------------------- clocks
 
 class ClockSampler:
@@ -115,17 +131,32 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def _size(self):
+        try:
+            return os.path.getsize(self.path)
+        except Exception:
+            return 0
+
+    def mark(self):
+        """Start of the timed regions: samples written before this point belong to the warm-up."""
+        self.begin = self._size()
+
     def stop(self):
         if self.proc is None:
             return None
         try:
+            time.sleep(0.05)                   # one more sampling period, so the last timed sample is on disk
             self.proc.terminate()
             self.proc.wait(timeout=5)
         except Exception:
             pass
         sm, smax, reasons = [], [], set()
         try:
-            for line in open(self.path):
+            data = open(self.path).read()
+            begin = getattr(self, "begin", 0)
+            # a sample that was being written when the region began or ended still counts
+            begin = data.rfind("\n", 0, begin) + 1
+            for line in data[begin:].splitlines():
                 f = [t.strip() for t in line.split(",")]
                 if len(f) < 9:
                     continue
@@ -142,7 +173,8 @@ class ClockSampler:
         if not sm:
             return None
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "period_ms": 20,
+                "covers": "the device-resident timed region and the end-to-end timed region that follows it"}
 
 
 # ---------------------------------------------------------------------------- our arm
@@ -152,9 +184,7 @@ def run_ours(args):
     import torch.distributed as dist
     from paper_2111_00153_b200 import binding as R
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
     torch.cuda.set_device(local)
@@ -249,6 +279,11 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # the clock sampler starts before the warm-up (nvidia-smi needs a moment to deliver its first line);
+    # its file position at the start of the timed region separates warm-up samples from timed ones
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
@@ -258,10 +293,9 @@ def run_ours(args):
     # ---- device-resident timing
     evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers]
            for _ in range(args.steps)]
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     barrier()
+    if rank == 0:
+        sampler.mark()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record(stream)
     for k in range(args.steps):
@@ -269,7 +303,6 @@ def run_ours(args):
     t1.record(stream)
     barrier()
     ms_total = t0.elapsed_time(t1)
-    clocks = sampler.stop() if rank == 0 else None
     ms_total = max_over_ranks(ms_total, world, "cuda")
     ms_step = ms_total / args.steps
     ops_step = sum(layer_ops(L, batch) for L in layers)
@@ -336,6 +369,7 @@ def run_ours(args):
         stream.wait_stream(s_out)
     t1.record(stream)
     barrier()
+    clocks = sampler.stop() if rank == 0 else None
     e2e_ms = max_over_ranks(t0.elapsed_time(t1), world, "cuda")
     e2e_ms_step = e2e_ms / max(e2e_steps, 1)
     h2d = int(sum(p["W"].numel() * 4 + p["x"].numel() * 4 for p in pin))
@@ -370,7 +404,7 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "tensor_kernel + pair_kernel (conv_implicit)", "achieved": achieved_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved_gbs / peaks["hbm_gbs"],
                      "peak_source": peak_src,
-                     "traffic": TRAFFIC_PER_STEP_BYTES if (batch == BATCH and use_ws and not args.layers) else None,
+                     "traffic": measured_traffic() if (batch == BATCH and use_ws and not args.layers) else None,
                      "algorithmic_bytes_per_step": float(alg.sum()), "kernel_ms_per_step": conv_total_ms,
                      "kernel_tops": ops_step / (conv_total_ms * 1e-3) / 1e12},
         "roofline_tensor": ({"bound": "tensor", "kernel": "pair_kernel (layers with K >= 2048 and M a multiple of 256)",
@@ -378,6 +412,7 @@ def run_ours(args):
                              "peak_source": "tcgen05.mma kind::i8 M=128 N=256 loop measured in this run (rmsmp_measure_mma_peak); "
                                             "2 x measured bf16 GEMM = %.0f" % (2 * peaks["bf16_tflops"]),
                              "layers": len(tb)} if tb and i8_peak > 0 else None),
+        "roofline_per_layer": binding_roof_summary(H, conv_ms_layer, alg, batch, peaks["hbm_gbs"], i8_peak, peaks),
         "per_layer": [{"name": h["L"].name, "M": h["L"].M, "K": h["L"].K, "N": d["N"], "ms": float(ms),
                        "tops": layer_ops(h["L"], batch) / (ms * 1e-3) / 1e12, "gbs": float(a / (ms * 1e-3) / 1e9)}
                       for h, d, ms, a in zip(H, D, conv_ms_layer, alg)],
@@ -389,10 +424,53 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# dram bytes (read + write) of the 19 convolution launches of one step at batch 256, from an ncu
-# capture of this kernel (profiles/bench_resnet18_stack_launch_list.md); reported only for that
-# configuration.  Set back to None whenever tensor_kernel changes.
-TRAFFIC_PER_STEP_BYTES = 1256.0e6
+def binding_roof_summary(H, ms_layer, alg_bytes, batch, hbm_gbs, i8_peak, peaks):
+    """Each convolution against its OWN binding roof: the roofline time of a layer is the larger of
+    bytes / HBM bandwidth and ops / INT8 tensor rate; the summary is sum(roofline time) / sum(time)."""
+    if not i8_peak or i8_peak <= 0:
+        return None
+    roof_ms, kinds = [], []
+    for h, a in zip(H, alg_bytes):
+        t_h = a / (hbm_gbs * 1e9) * 1e3
+        t_t = layer_ops(h["L"], batch) / (i8_peak * 1e12) * 1e3
+        roof_ms.append(max(t_h, t_t))
+        kinds.append("tensor" if t_t > t_h else "hbm")
+    tot = float(np.sum(ms_layer))
+    den = {"measured kind::i8 MMA loop": i8_peak, "2 x measured bf16 burst": 2 * peaks["bf16_tflops"],
+           "2 x measured bf16 sustained": 2 * peaks.get("bf16_tflops_sustained", 0.0), "datasheet dense int8": 4500.0}
+    tb = [(layer_ops(h["L"], batch), float(m)) for h, m, k in zip(H, ms_layer, kinds) if k == "tensor"]
+    t_tops = (sum(o for o, _ in tb) / (sum(m for _, m in tb) * 1e-3) / 1e12) if tb else None
+    return {"frac": float(np.sum(roof_ms)) / tot, "roofline_ms": float(np.sum(roof_ms)), "kernel_ms": tot,
+            "layers": [{"name": h["L"].name, "bound": k, "frac": float(r / m)} for h, k, r, m in zip(H, kinds, roof_ms, ms_layer)],
+            "tensor_bound_tops": t_tops,
+            "tensor_bound_frac_by_denominator": ({n: (t_tops / v if v else None) for n, v in den.items()} if t_tops else None)}
+
+
+TRAFFIC_NOTE = os.path.join(ROOT, "profiles", "resnet18_stack_dram_traffic.txt")
+KERNEL_SOURCES = ("tensor.cu", "tensor2.cu", "common.cuh", "decode.cuh", "actq.cuh")
+
+
+def kernel_sources_digest():
+    """sha256 over the sources of the convolution kernels: ties a counter capture to the code it measured."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2111_00153_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def measured_traffic():
+    """DRAM bytes (read + write) of the 19 convolution launches of one step at batch 256, as the
+    profiler's counters gave them, from the note the capture left -- or None when there is no note
+    or the kernels' sources have changed since (stale counters are not reported)."""
+    try:
+        kv = dict(line.split(":", 1) for line in open(TRAFFIC_NOTE) if ":" in line and not line.startswith("#"))
+        if kv["kernel_sources_sha256"].strip() != kernel_sources_digest():
+            return None
+        return float(kv["dram_bytes_per_step"])
+    except Exception:
+        return None
 
 
 def load_peaks():
@@ -400,10 +478,11 @@ def load_peaks():
     if os.path.exists(p):
         try:
             d = json.load(open(p))
-            return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"])}, "of measured"
+            return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                    "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", 0.0))}, "of measured"
         except Exception:
             pass
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "of fallback"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "of fallback"
 
 
 # ---------------------------------------------------------------------------- CPU oracle legs
@@ -461,6 +540,34 @@ def run_reference(args):
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def run_check_ranks(args):
+    """Plumbing self-check without a GPU (`--check-ranks`, any N): every rank joins a gloo group,
+    draws the first layer's weights and its own input batch, and the ranks compare checksums and
+    take the slowest of their (made-up) times.  Rank 0 prints what it found as one JSON line."""
+    import torch
+    import torch.distributed as dist
+    world, rank, _ = rank_env()
+    if world > 1:
+        dist.init_process_group("gloo")
+    L = synth.resnet18_convs()[-1]
+    W, x = host_layer(0, L, 2, rank)
+    mine = torch.tensor([float(np.abs(W).sum()), float(x.sum())], dtype=torch.float64)
+    every = [torch.zeros_like(mine) for _ in range(world)]
+    if world > 1:
+        dist.all_gather(every, mine)
+    else:
+        every = [mine]
+    ms = max_over_ranks(10.0 + 5.0 * rank, world, "cpu")
+    if rank == 0:
+        w = [float(t[0]) for t in every]
+        xs = [float(t[1]) for t in every]
+        print(json.dumps({"check": "ranks", "n_ranks": world, "weights_replicated": len(set(w)) == 1,
+                          "inputs_differ": len(set(xs)) == world, "max_ms": ms,
+                          "whole_job_tops_at_1e12_ops": whole_job_tops(10 ** 12, world, ms)}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 # ---------------------------------------------------------------------------- variant comparison
@@ -618,13 +725,19 @@ def main():
     ap.add_argument("--suite-filter", default=None,
                     help="with --suite: only the rows whose configuration tag contains this text "
                          "(config1 .. config5, or 'grouped' for the one-launch BERT-large stack)")
+    ap.add_argument("--check-ranks", action="store_true",
+                    help="no GPU work: the ranks check their seeding and the max-over-ranks exchange over gloo")
     ap.add_argument("--layers", default=None,
                     help="comma-separated layer names: run one instance of each (profiling runs)")
     args = ap.parse_args()
     if args.layers:
         global LAYER_FILTER
         LAYER_FILTER = set(args.layers.split(","))
-    if args.suite:
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.suite:
+        sys.exit(launch_ranks(sys.argv[1:], args.gpus))
+    if args.check_ranks:
+        run_check_ranks(args)
+    elif args.suite:
         run_suite(args)
     elif args.impl == "reference":
         run_reference(args)

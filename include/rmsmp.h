@@ -204,7 +204,7 @@ rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* layer, const void* d
 
 /*
  * Many small-batch linear layers in one launch (Algorithm 1's forward line, layer after layer;
- * Section 3.1: execution is "layer by layer on the same pieces of computing resource").  With a
+ * Section 3.1: the layers execute one after another on the same hardware).  With a
  * handful of tokens a layer is bound by reading its packed weights once, which takes a fraction
  * of a microsecond -- less than a kernel launch -- so the layers are handed over together and one
  * kernel streams all their weights.  Every item is computed exactly as rmsmp_gemm would (CUDA
@@ -294,12 +294,18 @@ rmsmp_status rmsmp_conv_implicit_workspace_requant(const rmsmp_layer* layer, con
  * Meant for code that runs under a runtime with a fixed memory arena, in a latency-critical
  * loop, or anywhere else cudaMalloc is off limits.
  *   - Limit: layer->M * layer->Kp <= 4 MiB (4,194,304 bytes), else RMSMP_ERR_BUFFER_TOO_SMALL.
+ *   - Only the tensor-core kernel is available here: a layer it cannot run (K or ld_act not a
+ *     multiple of 16) is refused with RMSMP_ERR_VARIANT instead of falling back to CUDA cores.
  *   - The first call on each device looks up the array's device address
- *     (cudaGetSymbolAddress); make that first call outside any stream capture.
+ *     (cudaGetSymbolAddress); with lazy module loading that lookup is also the moment the driver
+ *     places the array (and this library's kernels) on the device.  Make that first call during
+ *     set-up, outside any stream capture and before the memory budget is frozen.
  *   - All calls share the one array, and it keeps what the last call wrote.  Each call rewrites
  *     every byte it later reads, so stale contents are harmless, but two calls whose GPU work
  *     overlaps (different streams, or different host threads) race on it: serialise them.
- * Arguments and other errors: as rmsmp_gemm.
+ *   - Every argument is checked before anything is queued: a refused call leaves the array, and
+ *     any earlier call still running on it, untouched.
+ * Arguments and other errors: as rmsmp_gemm (NULL, BAD_LAYER, SHAPE, SCALE, ALIGN, ARCH, CUDA).
  */
 rmsmp_status rmsmp_gemm_builtin_scratch(const rmsmp_layer* layer, const void* d_packed,
                                         const int8_t* d_act, int64_t N, int64_t ld_act,

@@ -9,7 +9,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "librmsmp.so")
 SOURCES = ("host_api.cu", "pack.cu", "simt.cu", "tensor.cu", "tensor2.cu", "peak.cu", "builtin_scratch.cu")
-HEADERS = ("common.cuh", "decode.cuh", os.path.join("..", "..", "include", "rmsmp.h"))
+HEADERS = tuple(sorted(f for f in os.listdir(CSRC) if f.endswith((".cuh", ".h")))) + \
+          (os.path.join("..", "..", "include", "rmsmp.h"),)
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

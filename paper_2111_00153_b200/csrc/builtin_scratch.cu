@@ -8,6 +8,7 @@
 // the workspace variant needs lives in this file, in device memory that belongs to the loaded
 // library itself.
 #include <cuda_runtime.h>
+#include <atomic>
 #include "common.cuh"
 
 namespace {
@@ -20,26 +21,24 @@ static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratch
 
 // In host code `g_builtin_scratch` is only a handle for the runtime, not a device address; the
 // address each device gave the array is looked up once per device and kept here.
-void* g_scratch_ptr[64];
-bool g_scratch_known[64];
+// Host threads may make their first call on a device at the same time; the slot is an atomic pointer
+// (every thread that looks the address up gets the same answer, so a lost race costs one more lookup).
+std::atomic<void*> g_scratch_ptr[rmsmp::kMaxDevices];
 
 rmsmp_status scratch_address(void** out)
 {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
-        cudaGetLastError();
-        return RMSMP_ERR_CUDA;
-    }
-    if (!g_scratch_known[dev]) {
-        void* ptr = nullptr;
+    const int dev = rmsmp::device_ordinal();
+    if (dev < 0) return RMSMP_ERR_CUDA;
+    void* ptr = g_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
+        // With lazy module loading this lookup is also what makes the driver place the array on the device.
         if (cudaGetSymbolAddress(&ptr, g_builtin_scratch) != cudaSuccess || ptr == nullptr) {
             cudaGetLastError();
             return RMSMP_ERR_CUDA;
         }
-        g_scratch_ptr[dev] = ptr;
-        g_scratch_known[dev] = true;
+        g_scratch_ptr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_scratch_ptr[dev];
+    *out = ptr;
     return RMSMP_OK;
 }
 
@@ -58,10 +57,16 @@ extern "C" rmsmp_status rmsmp_gemm_builtin_scratch(const rmsmp_layer* layer, con
     void* scratch = nullptr;
     st = scratch_address(&scratch);
     if (st != RMSMP_OK) return st;
+    // Everything about the contraction is checked BEFORE the expansion is queued: a call that is going
+    // to be refused must not touch the shared array, which an earlier call's kernels may still be reading.
+    rmsmp::Problem p;
+    st = rmsmp::gemm_prepare(layer, d_packed, scratch, true, d_act, N, ld_act, act_step, d_out, ld_out, out_layout,
+                             d_acc, nullptr, p);
+    if (st != RMSMP_OK) return st;
+    if (!rmsmp::tensor_supported(p)) return RMSMP_ERR_VARIANT;
     // The expansion rewrites every byte the contraction will read (M rows of Kp bytes), so what an
     // earlier call left in the array never matters and nothing needs clearing.
     st = rmsmp_expand_weights(layer, d_packed, scratch, kBuiltinScratchBytes, stream);
     if (st != RMSMP_OK) return st;
-    return rmsmp_gemm_workspace(layer, d_packed, scratch, d_act, N, ld_act, act_step, d_out, ld_out,
-                                out_layout, d_acc, stream);
+    return rmsmp::dispatch_problem(p, RMSMP_VARIANT_TENSOR, static_cast<cudaStream_t>(stream));
 }

@@ -57,6 +57,33 @@ struct Problem {
     int64_t ld_codes;
 };
 
+// Per-device host state.  A process may drive several GPUs; anything learnt from or set on a device
+// (its SM count, a kernel's shared-memory attribute) is cached by the device's ordinal, never once
+// per process.  device_ordinal() returns the current device, or -1 when it cannot be had or lies
+// beyond the tables (kMaxDevices).
+constexpr int kMaxDevices = 64;
+int device_ordinal();
+int sm_count();               // SMs of the current device (cached per ordinal)
+// Calls cudaFuncSetAttribute(MaxDynamicSharedMemorySize) for `fn` once per device: `done` is the
+// kernel's own table of kMaxDevices flags.  Returns false if the attribute could not be set.
+bool ensure_smem_attr(const void* fn, int bytes, bool* done);
+
+// Re-quantizing epilogue request (rmsmp_*_workspace_requant): the next layer's clip value, kind and code buffer.
+struct Requant {
+    float alpha;
+    rmsmp_act_kind kind;
+    int8_t* codes;
+    int64_t ld;
+};
+
+// host side of the linear-layer calls, split so that a caller can validate before it queues anything
+// (host_api.cu): all checks + the problem description; then the launch of the chosen variant
+rmsmp_status gemm_prepare(const rmsmp_layer* L, const void* d_packed, const void* d_ws, bool use_ws,
+                          const int8_t* d_act, int64_t N, int64_t ld_act, float act_step, float* d_out,
+                          int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc, const Requant* rq,
+                          Problem& p);
+rmsmp_status dispatch_problem(Problem& p, rmsmp_variant variant, cudaStream_t st);
+
 // kernels (each returns the CUDA launch error, cudaSuccess if fine)
 cudaError_t launch_pack(const float* dW, int conv_oihw, const rmsmp_layer& L, int pot_mode,
                         uint8_t* blob, cudaStream_t st);

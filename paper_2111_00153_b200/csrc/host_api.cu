@@ -28,11 +28,10 @@ bool layer_ok(const rmsmp_layer* L)
 
 rmsmp_status check_arch()
 {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return RMSMP_ERR_CUDA; }
-    static int cached_major[64];
-    static bool have[64];
-    if (dev < 0 || dev >= 64) return RMSMP_ERR_CUDA;
+    const int dev = device_ordinal();
+    static int cached_major[kMaxDevices];
+    static bool have[kMaxDevices];
+    if (dev < 0) return RMSMP_ERR_CUDA;
     if (!have[dev]) {
         int major = 0;
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
@@ -64,15 +63,15 @@ struct StageRing {
     bool used[kStageSlots];
     int next = 0;
 };
-StageRing g_stage[64];
+StageRing g_stage[kMaxDevices];
 std::mutex g_stage_mutex;
 
 // Copies `bytes` of metadata to the device through a pinned slot; false = caller uses the pageable path.
 bool staged_upload(void* d_dst, const void* h_src, size_t bytes, cudaStream_t st)
 {
     if (bytes > kStageSlotBytes) return false;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return false; }
+    const int dev = device_ordinal();
+    if (dev < 0) return false;
     std::lock_guard<std::mutex> lock(g_stage_mutex);
     StageRing& r = g_stage[dev];
     if (!r.tried) {
@@ -147,6 +146,44 @@ rmsmp_status dispatch(Problem& p, rmsmp_variant variant, cudaStream_t st)
 }
 
 }  // namespace
+
+namespace rmsmp {
+
+int device_ordinal()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
+    return (dev >= 0 && dev < kMaxDevices) ? dev : -1;
+}
+
+int sm_count()
+{
+    static int cached[kMaxDevices];
+    const int dev = device_ordinal();
+    if (dev < 0) return 1;
+    if (cached[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) cudaGetLastError();
+        cached[dev] = v > 0 ? v : 1;
+    }
+    return cached[dev];
+}
+
+bool ensure_smem_attr(const void* fn, int bytes, bool* done)
+{
+    const int dev = device_ordinal();
+    if (dev < 0) return false;
+    if (!done[dev]) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        done[dev] = true;
+    }
+    return true;
+}
+
+}  // namespace rmsmp
 
 extern "C" {
 
@@ -345,14 +382,6 @@ rmsmp_status rmsmp_quantize_act(const float* d_X, size_t count, float alpha_a, r
     return RMSMP_OK;
 }
 
-// Re-quantizing epilogue request (rmsmp_*_workspace_requant): the next layer's clip value, kind and code buffer.
-struct Requant {
-    float alpha;
-    rmsmp_act_kind kind;
-    int8_t* codes;
-    int64_t ld;
-};
-
 static rmsmp_status requant_check(const Requant* rq, float* h_next_step)
 {
     if (!rq->codes) return RMSMP_ERR_NULL;
@@ -362,10 +391,16 @@ static rmsmp_status requant_check(const Requant* rq, float* h_next_step)
     return RMSMP_OK;
 }
 
-static rmsmp_status gemm_impl(const rmsmp_layer* L, const void* d_packed, const void* d_ws, bool use_ws,
-                              const int8_t* d_act, int64_t N, int64_t ld_act, float act_step, float* d_out,
-                              int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
-                              rmsmp_variant variant, void* stream, const Requant* rq = nullptr)
+}  // extern "C"
+
+namespace rmsmp {
+
+// Every host-side check of a linear-layer call, and the kernel's problem description.  Nothing is
+// launched here, so a caller can validate first and queue work only for calls that will go through.
+rmsmp_status gemm_prepare(const rmsmp_layer* L, const void* d_packed, const void* d_ws, bool use_ws,
+                          const int8_t* d_act, int64_t N, int64_t ld_act, float act_step, float* d_out,
+                          int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc, const Requant* rq,
+                          Problem& p)
 {
     if (!L || !d_packed || !d_act || (!d_out && !rq) || (use_ws && !d_ws)) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
@@ -378,9 +413,9 @@ static rmsmp_status gemm_impl(const rmsmp_layer* L, const void* d_packed, const 
     if (!aligned16(d_act) || (!rq && !aligned16(d_out)) || (d_acc && !aligned16(d_acc)) || (ld_act & 15) ||
         (reinterpret_cast<uintptr_t>(d_packed) & 255))
         return RMSMP_ERR_ALIGN;
+    if (use_ws && !aligned16(d_ws)) return RMSMP_ERR_ALIGN;
     rmsmp_status a = check_arch();
     if (a != RMSMP_OK) return a;
-    Problem p;
     fill_problem(p, L, d_packed);
     p.act = d_act;
     p.B = (int)std::min<int64_t>(N, 0x7fffffff); p.H = 1; p.W = 1; p.Ho = 1; p.Wo = 1; p.stride = 1; p.pad = 0;
@@ -388,12 +423,27 @@ static rmsmp_status gemm_impl(const rmsmp_layer* L, const void* d_packed, const 
     p.act_step = act_step; p.out = d_out; p.acc = d_acc; p.ld_out = ld_out;
     p.out_mn = (out_layout == RMSMP_OUT_MN);
     if (rq) { p.rq_codes = rq->codes; p.rq_alpha = rq->alpha; p.rq_kind = rq->kind; p.ld_codes = rq->ld; }
-    if (use_ws) {
-        if (!aligned16(d_ws)) return RMSMP_ERR_ALIGN;
-        p.wexp = static_cast<const int8_t*>(d_ws);
-    }
+    if (use_ws) p.wexp = static_cast<const int8_t*>(d_ws);
+    return RMSMP_OK;
+}
+
+rmsmp_status dispatch_problem(Problem& p, rmsmp_variant variant, cudaStream_t st) { return dispatch(p, variant, st); }
+
+}  // namespace rmsmp
+
+static rmsmp_status gemm_impl(const rmsmp_layer* L, const void* d_packed, const void* d_ws, bool use_ws,
+                              const int8_t* d_act, int64_t N, int64_t ld_act, float act_step, float* d_out,
+                              int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
+                              rmsmp_variant variant, void* stream, const Requant* rq = nullptr)
+{
+    Problem p;
+    rmsmp_status s = gemm_prepare(L, d_packed, d_ws, use_ws, d_act, N, ld_act, act_step, d_out, ld_out, out_layout,
+                                  d_acc, rq, p);
+    if (s != RMSMP_OK) return s;
     return dispatch(p, variant, static_cast<cudaStream_t>(stream));
 }
+
+extern "C" {
 
 rmsmp_status rmsmp_grouped_table_bytes(int count, size_t* bytes)
 {

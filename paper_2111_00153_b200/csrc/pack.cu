@@ -219,7 +219,8 @@ cudaError_t launch_unpack(const rmsmp_layer& L, const uint8_t* blob, int8_t* val
                           int32_t* perm, float* wstep, cudaStream_t st)
 {
     int64_t total = (int64_t)L.M * L.Cin * L.kh * L.kw;
-    int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    const int64_t cap = (int64_t)sm_count() * 16;
+    int blocks = (int)((total + 255) / 256 < cap ? (total + 255) / 256 : cap);
     unpack_kernel<<<blocks, 256, 0, st>>>(blob, L, values, perm, wstep);
     return cudaGetLastError();
 }
@@ -271,7 +272,7 @@ cudaError_t launch_expand(const rmsmp_layer& L, const uint8_t* blob, int8_t* wex
 {
     const int64_t total = (int64_t)L.M * (L.Kp >> 5);
     int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
     expand_kernel<<<(unsigned)blocks, 256, 0, st>>>(blob, L, wexp);
     return cudaGetLastError();
 }
@@ -345,7 +346,7 @@ cudaError_t launch_quantize_act(const float* x, size_t count, float alpha, int k
     int vec = ((reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(codes) & 15) == 0);
     size_t steps = vec ? (count + 31) / 32 : count;      // the vector path handles 32 values per thread and step
     size_t blocks = (steps + 255) / 256;
-    const size_t cap = 148 * 32;
+    const size_t cap = (size_t)sm_count() * 32;
     if (blocks > cap) blocks = cap;
     if (blocks == 0) blocks = 1;
     quantize_act_kernel<<<(unsigned)blocks, 256, 0, st>>>(x, count, alpha, kind, codes, vec);

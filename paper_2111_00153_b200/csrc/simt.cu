@@ -54,7 +54,7 @@ cudaError_t launch_simple(const Problem& p, cudaStream_t st)
 {
     int64_t total = p.N * p.M;
     int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 64) blocks = 148 * 64;
+    if (blocks > (int64_t)sm_count() * 64) blocks = (int64_t)sm_count() * 64;
     simple_kernel<<<(unsigned)blocks, 256, 0, st>>>(p);
     return cudaGetLastError();
 }
@@ -189,7 +189,7 @@ cudaError_t launch_simt(const Problem& p, bool shiftadd, cudaStream_t st)
     const int64_t ngroups = (p.N + kTok - 1) / kTok;
     int64_t warps = ngroups * p.M;
     int64_t blocks = (warps + 7) / 8;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
     if (shiftadd) rowwarp_kernel<true><<<(unsigned)blocks, 256, 0, st>>>(p);
     else rowwarp_kernel<false><<<(unsigned)blocks, 256, 0, st>>>(p);
     return cudaGetLastError();
@@ -603,7 +603,7 @@ int grouped_fill_table(const Problem* probs, int count, uint8_t* h_table)
 cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t total, int nt, cudaStream_t st)
 {
     int64_t blocks = (total + 7) / 8;
-    if (blocks > 148 * 2) blocks = 148 * 2;                  // one resident wave: two blocks of 128-register threads per SM
+    if (blocks > (int64_t)sm_count() * 2) blocks = (int64_t)sm_count() * 2;                  // one resident wave: two blocks of 128-register threads per SM
     if (blocks < 1) blocks = 1;
     const int use_smem = table_bytes <= (size_t)kGroupedSmemMax;
     const size_t smem = use_smem ? table_bytes : 0;

@@ -936,18 +936,6 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-int sm_count()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) cudaGetLastError();
-        n = v > 0 ? v : 148;
-    }
-    return n;
-}
-
 // Tensor maps of the activation codes for boxes of `bk` channels x th output rows x tb images
 // (see act_parity_split: one map, or one per parity sub-grid of a stride-2 layer).
 bool encode_act_maps(EncodeTiledFn enc, const Problem& p, int bk, int th, int tb, CUtensorMapSwizzle swz, CUtensorMap out[4])
@@ -1194,14 +1182,8 @@ rmsmp_status launch_tensor(const Problem& p, cudaStream_t st)
     const int io = p.rq_codes ? 1 : ((c.tma_store && !p.out_mn && !p.acc) ? 2 : 0);
     const KernelFn fn = table[mode][i2][io];
     if (!fn) return RMSMP_ERR_VARIANT;
-    static bool attr_set[4][2][3] = {};
-    if (!attr_set[mode][i2][io]) {
-        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
-            cudaGetLastError();
-            return RMSMP_ERR_CUDA;
-        }
-        attr_set[mode][i2][io] = true;
-    }
+    static bool attr_set[4][2][3][kMaxDevices] = {};
+    if (!ensure_smem_attr(reinterpret_cast<const void*>(fn), kSmemLimit, attr_set[mode][i2][io])) return RMSMP_ERR_CUDA;
     const int grid = (int)std::min<int64_t>(c.ntiles, sm_count());
     fn<<<grid, kThreads, c.smem_bytes, st>>>(p, c, mp);
     if (cudaGetLastError() != cudaSuccess) return RMSMP_ERR_CUDA;

@@ -412,18 +412,6 @@ EncodeTiledFn2 encode_fn2()
     return fn;
 }
 
-int sm_count2()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) cudaGetLastError();
-        n = v > 0 ? v : 148;
-    }
-    return n;
-}
-
 // The pair kernel takes: expanded weights, an even number of row blocks, full 128-channel chunks,
 // fp32 [N][M] output through bulk stores, no accumulator dump, no re-quantizing epilogue.
 bool plan_pair(const Problem& p, PairCfg& c)
@@ -505,15 +493,9 @@ rmsmp_status launch_pair(const Problem& p, cudaStream_t st)
     if (!make_out(&mp.out_full, 32)) return RMSMP_ERR_CUDA;
     if (c.tail_rows && !make_out(&mp.out_tail, c.tail_rows)) return RMSMP_ERR_CUDA;
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem_bytes) != cudaSuccess) {
-            cudaGetLastError();
-            return RMSMP_ERR_CUDA;
-        }
-        attr_set = true;
-    }
-    const int clusters = (int)std::min<int64_t>(c.ntiles, sm_count2() / 2);
+    static bool attr_set[kMaxDevices] = {};
+    if (!ensure_smem_attr(reinterpret_cast<const void*>(pair_kernel), (int)c.smem_bytes, attr_set)) return RMSMP_ERR_CUDA;
+    const int clusters = (int)std::min<int64_t>(c.ntiles, sm_count() / 2);
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof(lc));
     lc.gridDim = dim3((unsigned)(2 * clusters), 1, 1);

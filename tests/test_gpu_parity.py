@@ -372,6 +372,95 @@ def test_conv_requant_epilogue(M, Cin, k, stride, pad, B, H, W, kind):
     assert np.array_equal(out.cpu().numpy(), want)
 
 
+def _ulps(x, n):
+    """fp32 value n units in the last place away from x."""
+    v = np.float32(x)
+    for _ in range(abs(n)):
+        v = np.nextafter(v, np.float32(np.inf if n > 0 else -np.inf), dtype=np.float32)
+    return v
+
+
+@pytest.mark.parametrize("kind", [R.ACT_U4, R.ACT_S4])
+@pytest.mark.parametrize("M,ld_extra", [(128, 0), (130, 14), (64, 0)], ids=["bulk", "direct", "dup"])
+@pytest.mark.parametrize("step_ulps", [0, 1, -1, 4, -4])
+def test_requant_epilogue_on_rounding_boundaries(M, ld_extra, step_ulps, kind):
+    """The fused quantizer exactly ON, and a few units in the last place either side of, its
+    rounding boundaries.  All rows are Fixed-8 with alpha = 127, so wstep = 1 and the weights are
+    the integers they are given as; with act_step = 1 the layer output y equals the integer sum.
+    next_alpha is chosen so that y / next_alpha * Q = y / 2: every odd sum lies exactly on a
+    half-level (the tie goes to the even code), and an act_step a few ulps off 1 moves every value
+    just off its level or half-level.  Expected codes: the oracle's epilogue followed by the
+    oracle's quantizer, so its chain of fp32 roundings decides."""
+    import torch
+    K, N = 64, 700
+    g = synth.rng(83, M + step_ulps + 10 * kind)
+    lo = 0 if kind == R.ACT_U4 else -1
+    Wt = g.integers(lo, 2, size=(M, K)).astype(np.float32)          # values in {0, 1} (U4) or {-1, 0, 1} (S4)
+    Wt[g.random((M, K)) < (0.93 if kind == R.ACT_U4 else 0.8)] = 0.0  # sums of a few codes: mostly inside the clip range
+    Wt[:, 0] = 127.0                                                  # one full-scale entry per row keeps the values exact ...
+    scheme = np.ones(M, np.uint8)
+    bits = np.full(M, 8, np.uint8)
+    alpha = np.full(M, 127.0, np.float32)
+    codes = synth.act_codes_uniform(g, (N, K))
+    codes[:, 0] = 0                                                   # ... and never contributes to a sum
+    if kind == R.ACT_S4:
+        codes = (codes % 15 - 7).astype(np.int8)
+        codes[:, 0] = 0
+    act_step = _ulps(1.0, step_ulps)
+    na = 30.0 if kind == R.ACT_U4 else 14.0
+    values, wstep, acc_ref, y_ref = O.layer_linear(Wt, scheme, bits, alpha, codes, act_step)
+    assert np.all(wstep == np.float32(1.0)) and np.array_equal(values, Wt.astype(np.int8))
+    odd = (np.abs(acc_ref) % 2 == 1) & (np.abs(acc_ref) < 30)
+    assert odd.mean() > 0.25                                           # a large share of outputs sits on a half-level
+    want, _ = O.quantize_act(y_ref, na, kind)
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(layer, d_packed, ws)
+    ld = M + ld_extra
+    out = torch.full((N, ld), 99, dtype=torch.int8, device="cuda")
+    R.rmsmp_gemm_workspace_requant(layer, d_packed, ws, torch.from_numpy(codes).cuda(), N, K, float(act_step),
+                                   na, kind, out, ld)
+    torch.cuda.synchronize()
+    assert R.rmsmp_last_device_status(d_packed) == R.OK
+    got = out.cpu().numpy()
+    assert np.array_equal(got[:, :M], want)
+    assert (got[:, M:] == 99).all()
+    if step_ulps == 0:
+        # with exact halves the expected code is the even neighbour, by the definition alone
+        q = 15 if kind == R.ACT_U4 else 7
+        t = np.clip(acc_ref.astype(np.float64) / na, 0.0 if kind == R.ACT_U4 else -1.0, 1.0) * q
+        assert np.array_equal(want, np.rint(t).astype(np.int8))
+
+
+def test_conv_requant_epilogue_on_rounding_boundaries():
+    """The same construction through the convolution kernel's resident-weight form (3x3, 64 channels)."""
+    import torch
+    M, Cin, k, B, H = 64, 64, 3, 2, 12
+    g = synth.rng(83, 999)
+    Wt = g.integers(0, 2, size=(M, Cin, k, k)).astype(np.float32)
+    Wt[g.random(Wt.shape) < 0.992] = 0.0
+    Wt[:, 0, 0, 0] = 127.0
+    scheme = np.ones(M, np.uint8)
+    bits = np.full(M, 8, np.uint8)
+    alpha = np.full(M, 127.0, np.float32)
+    codes = synth.act_codes_uniform(g, (B, H, H, Cin))
+    codes[..., 0] = 0
+    for ulps in (0, 2, -2):
+        act_step = _ulps(1.0, ulps)
+        _, _, acc_ref, y_ref = O.layer_conv(Wt, scheme, bits, alpha, codes, act_step, 1, 1)
+        assert ((acc_ref % 2 == 1) & (acc_ref < 30)).mean() > 0.2
+        want, _ = O.quantize_act(y_ref.reshape(-1, M), 30.0, O.ACT_U4)
+        layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+        ws = torch.empty(R.rmsmp_workspace_bytes(layer), dtype=torch.int8, device="cuda")
+        R.rmsmp_expand_weights(layer, d_packed, ws)
+        out = torch.full(want.shape, 99, dtype=torch.int8, device="cuda")
+        R.rmsmp_conv_implicit_workspace_requant(layer, d_packed, ws, torch.from_numpy(codes).cuda(), B, H, H, 1, 1,
+                                                float(act_step), 30.0, R.ACT_U4, out)
+        torch.cuda.synchronize()
+        assert R.rmsmp_last_device_status(d_packed) == R.OK
+        assert np.array_equal(out.cpu().numpy(), want)
+
+
 def test_requant_rejects_bad_arguments():
     import torch
     g = synth.rng(83)

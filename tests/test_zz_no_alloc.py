@@ -4,12 +4,14 @@ Some callers of the library may not allocate device memory when they call it (a 
 a runtime with a fixed arena, a latency-critical loop); for them the scratch of the workspace
 variant is an array inside the library.  The test runs the entry point twice in a row through
 the C ABI -- a large layer first, then a smaller one, so the second call finds the first call's
-bytes still in the shared array -- and requires the same bits as the caller-scratch path.
-This file is collected last on purpose.
+bytes still in the shared array -- and requires the same bits as the caller-scratch path and
+as the CPU oracle's linear layer.  A call that is refused (bad argument, shape the tensor kernel
+cannot run) must not have touched the array.  This file is collected last on purpose.
 """
 import numpy as np
 import pytest
 
+from oracle import rmsmp_oracle as O
 from paper_2111_00153_b200 import binding as R
 from paper_2111_00153_b200 import synth
 from tests import harness as Hn
@@ -41,6 +43,9 @@ def _run(M, K, N, seed):
     assert R.rmsmp_last_device_status(d_packed) == R.OK
     assert torch.equal(acc, acc_ref)
     assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.cpu().numpy().view(np.uint32))
+    _, _, acc_o, y_o = O.layer_linear(W, scheme, bits, alpha, act, np.float32(step))
+    assert np.array_equal(acc.cpu().numpy(), acc_o)
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), y_o.view(np.uint32))
 
 
 def test_two_calls_in_a_row_match_the_workspace_path():
@@ -58,3 +63,35 @@ def test_layer_beyond_the_built_in_scratch_is_rejected():
     with pytest.raises(R.RmsmpError) as e:
         R.rmsmp_gemm_builtin_scratch(layer, buf, buf, 16, K, 1.0, buf, M)
     assert e.value.status == R.ERR_BUFFER_TOO_SMALL
+
+
+def test_refused_calls_leave_the_shared_array_alone():
+    """A good call, then calls that must be refused before anything is queued, then the good call
+    again: the refusals return their documented codes and the repeated call is still bit-exact."""
+    import torch
+    _run(256, 512, 64, 3)
+    # K = 40 is not a multiple of 16: only the tensor-core kernel exists behind this entry point
+    g = synth.rng(80, 4)
+    W = synth.weights_normal(g, (64, 40))
+    scheme, bits = R.rmsmp_assign_rows(W, synth.RATIO_RMSMP1)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, synth.alpha_rows(W))
+    a = torch.zeros((8, 48), dtype=torch.int8, device="cuda")
+    y = torch.zeros((8, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_builtin_scratch(layer, d_packed, a, 8, 48, 0.1, y, 64)
+    assert e.value.status == R.ERR_VARIANT
+    # output leading dimension smaller than M, and a misaligned activation pointer
+    g = synth.rng(80, 5)
+    W = synth.weights_normal(g, (128, 256))
+    scheme, bits = R.rmsmp_assign_rows(W, synth.RATIO_RMSMP1)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, synth.alpha_rows(W))
+    a = torch.zeros((8 * 256 + 16,), dtype=torch.int8, device="cuda")
+    y = torch.zeros((8, 128), dtype=torch.float32, device="cuda")
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_builtin_scratch(layer, d_packed, a, 8, 256, 0.1, y, 64)
+    assert e.value.status == R.ERR_SHAPE
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_builtin_scratch(layer, d_packed, a[1:], 8, 256, 0.1, y, 128)
+    assert e.value.status == R.ERR_ALIGN
+    torch.cuda.synchronize()
+    _run(256, 512, 64, 3)
