@@ -231,6 +231,44 @@ rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp
                                 void* d_table, size_t table_bytes, void* stream);
 
 /*
+ * The same grouped launch on the tensor cores, split into a set-up call and a launch call
+ * (Section 3.1: rows of every scheme streamed to their cores and finishing together; here all
+ * layers' packed rows stream through the SMs in one kernel).  One persistent CTA per SM takes
+ * blocks of 128 rows of any layer, fetches their packed codes with TMA, expands them to int8 in
+ * shared memory and multiplies them with up to 256 tokens on tcgen05 (int32 accumulators in
+ * tensor memory).  Results are bit for bit those of rmsmp_gemm.
+ *   rmsmp_grouped_plan_bytes    scratch size for the table of these layers on the current device.
+ *   rmsmp_gemm_grouped_prepare  validates the items, builds the table (tensor maps of every
+ *                               layer's packed rows and activations, work lists per SM) and queues
+ *                               its upload to d_table (256-byte aligned) on `stream`; fills *plan.
+ *                               Every item needs N <= 128; more tokens (up to 256) are taken while
+ *                               the stages still fit shared memory, else RMSMP_ERR_VARIANT.  The call
+ *                               costs host time proportional to the number of layers: do it once.
+ *   rmsmp_gemm_grouped_launch   one kernel launch from a prepared plan; may be repeated for as
+ *                               long as the buffers, shapes and leading dimensions the plan was
+ *                               built from stay the same (their CONTENTS may change: new weights
+ *                               packed with the same row map, new activation codes).  The table
+ *                               must stay untouched while launches that use it are in flight.
+ * Errors: as rmsmp_gemm_grouped; BAD_LAYER for a plan that was not prepared, or was prepared on
+ * another device.
+ */
+typedef struct rmsmp_grouped_plan {
+    uint32_t magic;            /* set by rmsmp_gemm_grouped_prepare */
+    int32_t count;             /* layers */
+    int32_t grid;              /* CTAs of the launch */
+    uint32_t smem_bytes;       /* dynamic shared memory per CTA */
+    int32_t device;            /* ordinal of the device the table was built for */
+    int32_t reserved;
+    const void* d_table;
+    uint64_t table_bytes;
+} rmsmp_grouped_plan;
+rmsmp_status rmsmp_grouped_plan_bytes(const rmsmp_gemm_item* h_items, int count, size_t* bytes);
+rmsmp_status rmsmp_gemm_grouped_prepare(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
+                                        void* d_table, size_t table_bytes, rmsmp_grouped_plan* plan,
+                                        void* stream);
+rmsmp_status rmsmp_gemm_grouped_launch(const rmsmp_grouped_plan* plan, void* stream);
+
+/*
  * Workspace variant of the tensor-core path.  The expansion of the 4-bit / PoT codes to int8
  * (the GPU counterpart of routing rows to the per-scheme GEMM cores, Section 4.1) is done ONCE
  * per layer into caller-provided scratch memory instead of once per output tile in shared

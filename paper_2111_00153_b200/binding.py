@@ -32,6 +32,7 @@ EXPORTS = (
     "rmsmp_measure_mma_peak", "rmsmp_workspace_bytes", "rmsmp_expand_weights", "rmsmp_gemm_workspace",
     "rmsmp_conv_implicit_workspace", "rmsmp_gemm_builtin_scratch", "rmsmp_grouped_table_bytes",
     "rmsmp_gemm_grouped", "rmsmp_gemm_workspace_requant", "rmsmp_conv_implicit_workspace_requant",
+    "rmsmp_grouped_plan_bytes", "rmsmp_gemm_grouped_prepare", "rmsmp_gemm_grouped_launch",
 )
 
 
@@ -58,6 +59,13 @@ class rmsmp_gemm_item(C.Structure):
         ("layer", C.POINTER(rmsmp_layer)), ("d_packed", C.c_void_p), ("d_act", C.c_void_p),
         ("N", C.c_int64), ("ld_act", C.c_int64), ("act_step", C.c_float),
         ("d_out", C.c_void_p), ("ld_out", C.c_int64), ("d_acc", C.c_void_p),
+    ]
+
+
+class rmsmp_grouped_plan(C.Structure):
+    _fields_ = [
+        ("magic", C.c_uint32), ("count", C.c_int32), ("grid", C.c_int32), ("smem_bytes", C.c_uint32),
+        ("device", C.c_int32), ("reserved", C.c_int32), ("d_table", C.c_void_p), ("table_bytes", C.c_uint64),
     ]
 
 
@@ -105,6 +113,10 @@ def lib() -> C.CDLL:
         L.rmsmp_gemm_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
         L.rmsmp_grouped_table_bytes.argtypes = [i32, C.POINTER(C.c_size_t)]
         L.rmsmp_gemm_grouped.argtypes = [C.POINTER(rmsmp_gemm_item), i32, i32, vp, C.c_size_t, vp]
+        L.rmsmp_grouped_plan_bytes.argtypes = [C.POINTER(rmsmp_gemm_item), i32, C.POINTER(C.c_size_t)]
+        L.rmsmp_gemm_grouped_prepare.argtypes = [C.POINTER(rmsmp_gemm_item), i32, i32, vp, C.c_size_t,
+                                                 C.POINTER(rmsmp_grouped_plan), vp]
+        L.rmsmp_gemm_grouped_launch.argtypes = [C.POINTER(rmsmp_grouped_plan), vp]
         L.rmsmp_gemm_builtin_scratch.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i64, i64, f32, vp, i64, i32, vp, vp]
         L.rmsmp_conv_implicit_workspace.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
                                                     f32, vp, i32, vp, vp]
@@ -311,6 +323,26 @@ def rmsmp_gemm_grouped(items_array, out_layout: int, d_table, table_bytes: int |
         table_bytes = d_table.numel() * d_table.element_size()
     _check(lib().rmsmp_gemm_grouped(items_array, len(items_array), out_layout, _dp(d_table), table_bytes,
                                     _stream(stream)), "rmsmp_gemm_grouped")
+
+
+def rmsmp_grouped_plan_bytes(items_array) -> int:
+    n = C.c_size_t(0)
+    _check(lib().rmsmp_grouped_plan_bytes(items_array, len(items_array), C.byref(n)), "rmsmp_grouped_plan_bytes")
+    return n.value
+
+
+def rmsmp_gemm_grouped_prepare(items_array, out_layout: int, d_table, table_bytes: int | None = None, stream=None):
+    """Builds the tensor-core grouped launch of these layers into d_table; returns the plan to launch."""
+    if table_bytes is None:
+        table_bytes = d_table.numel() * d_table.element_size()
+    plan = rmsmp_grouped_plan()
+    _check(lib().rmsmp_gemm_grouped_prepare(items_array, len(items_array), out_layout, _dp(d_table), table_bytes,
+                                            C.byref(plan), _stream(stream)), "rmsmp_gemm_grouped_prepare")
+    return plan
+
+
+def rmsmp_gemm_grouped_launch(plan, stream=None):
+    _check(lib().rmsmp_gemm_grouped_launch(C.byref(plan), _stream(stream)), "rmsmp_gemm_grouped_launch")
 
 
 def rmsmp_last_device_status(d_packed, stream=None) -> int:

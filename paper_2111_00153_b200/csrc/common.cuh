@@ -99,6 +99,13 @@ cudaError_t launch_simt(const Problem& p, bool shiftadd, cudaStream_t st);
 size_t grouped_table_bytes(int count);
 int grouped_fill_table(const Problem* probs, int count, uint8_t* h_table);
 cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t total, int nt, cudaStream_t st);
+// grouped tensor-core launch (stream.cu): table size, per-problem support test, host-side table and
+// launch geometry, launch
+size_t stream_table_bytes(int count, int64_t nitems, int sms);
+bool stream_supported(const Problem& p);
+bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_table, size_t table_bytes,
+                        int* grid_out, uint32_t* smem_out);
+cudaError_t launch_stream(const uint8_t* d_table, int grid, uint32_t smem_bytes, cudaStream_t st);
 // returns false if the tensor variant cannot run this problem (alignment / shape)
 bool tensor_supported(const Problem& p);
 rmsmp_status launch_tensor(const Problem& p, cudaStream_t st);

@@ -12,6 +12,8 @@ namespace {
 
 inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
+constexpr uint32_t kPlanMagicHost = 0x47504C4Eu;   // "GPLN": rmsmp_grouped_plan filled by rmsmp_gemm_grouped_prepare
+
 inline int row_kind(int scheme, int bits)
 {
     if (scheme == RMSMP_SCHEME_POT && bits == 4) return kPoT4;
@@ -453,15 +455,14 @@ rmsmp_status rmsmp_grouped_table_bytes(int count, size_t* bytes)
     return RMSMP_OK;
 }
 
-rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
-                                void* d_table, size_t table_bytes, void* stream)
+// Host checks of a grouped call's items and their problem descriptions (nothing is launched).
+static rmsmp_status grouped_problems(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
+                                     std::vector<Problem>& probs)
 {
-    if (!h_items || !d_table) return RMSMP_ERR_NULL;
+    if (!h_items) return RMSMP_ERR_NULL;
     if (count < 1 || count > 65536) return RMSMP_ERR_SHAPE;
     if (out_layout != RMSMP_OUT_NM && out_layout != RMSMP_OUT_MN) return RMSMP_ERR_SHAPE;
-    if (table_bytes < grouped_table_bytes(count)) return RMSMP_ERR_BUFFER_TOO_SMALL;
-    if (!aligned16(d_table)) return RMSMP_ERR_ALIGN;
-    std::vector<Problem> probs((size_t)count);
+    probs.resize((size_t)count);
     for (int i = 0; i < count; ++i) {
         const rmsmp_gemm_item& it = h_items[i];
         const rmsmp_layer* L = it.layer;
@@ -482,6 +483,18 @@ rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp
         p.act_step = it.act_step; p.out = it.d_out; p.acc = it.d_acc; p.ld_out = it.ld_out;
         p.out_mn = (out_layout == RMSMP_OUT_MN);
     }
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
+                                void* d_table, size_t table_bytes, void* stream)
+{
+    if (!d_table) return RMSMP_ERR_NULL;
+    std::vector<Problem> probs;
+    rmsmp_status s = grouped_problems(h_items, count, out_layout, probs);
+    if (s != RMSMP_OK) return s;
+    if (table_bytes < grouped_table_bytes(count)) return RMSMP_ERR_BUFFER_TOO_SMALL;
+    if (!aligned16(d_table)) return RMSMP_ERR_ALIGN;
     rmsmp_status a = check_arch();
     if (a != RMSMP_OK) return a;
     std::vector<uint8_t> table(grouped_table_bytes(count));
@@ -495,6 +508,77 @@ rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp
         return RMSMP_ERR_CUDA;
     }
     if (launch_grouped(static_cast<const uint8_t*>(d_table), table.size(), total, nt, st) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return RMSMP_OK;
+}
+
+static int64_t grouped_row_blocks(const rmsmp_gemm_item* h_items, int count)
+{
+    int64_t n = 0;
+    for (int i = 0; i < count; ++i) n += h_items[i].layer ? h_items[i].layer->nblocks : 0;
+    return n;
+}
+
+rmsmp_status rmsmp_grouped_plan_bytes(const rmsmp_gemm_item* h_items, int count, size_t* bytes)
+{
+    if (!h_items || !bytes) return RMSMP_ERR_NULL;
+    if (count < 1 || count > 65536) return RMSMP_ERR_SHAPE;
+    for (int i = 0; i < count; ++i) {
+        if (!h_items[i].layer) return RMSMP_ERR_NULL;
+        if (!layer_ok(h_items[i].layer)) return RMSMP_ERR_BAD_LAYER;
+    }
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    *bytes = stream_table_bytes(count, grouped_row_blocks(h_items, count), sm_count());
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_gemm_grouped_prepare(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
+                                        void* d_table, size_t table_bytes, rmsmp_grouped_plan* plan, void* stream)
+{
+    if (!d_table || !plan) return RMSMP_ERR_NULL;
+    std::memset(plan, 0, sizeof(*plan));
+    std::vector<Problem> probs;
+    rmsmp_status s = grouped_problems(h_items, count, out_layout, probs);
+    if (s != RMSMP_OK) return s;
+    if ((reinterpret_cast<uintptr_t>(d_table) & 255) != 0) return RMSMP_ERR_ALIGN;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    for (const Problem& p : probs)
+        if (!stream_supported(p)) return RMSMP_ERR_VARIANT;
+    const size_t need = stream_table_bytes(count, grouped_row_blocks(h_items, count), sm_count());
+    if (table_bytes < need) return RMSMP_ERR_BUFFER_TOO_SMALL;
+    std::vector<uint8_t> table(need);
+    int grid = 0;
+    uint32_t smem = 0;
+    if (!stream_build_table(probs.data(), count, sm_count(), table.data(), need, &grid, &smem)) return RMSMP_ERR_VARIANT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the table leaves from pageable memory: the copy has read it when the call returns
+    if (cudaMemcpyAsync(d_table, table.data(), need, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    plan->magic = kPlanMagicHost;
+    plan->count = count;
+    plan->grid = grid;
+    plan->smem_bytes = smem;
+    plan->device = device_ordinal();
+    plan->d_table = d_table;
+    plan->table_bytes = need;
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_gemm_grouped_launch(const rmsmp_grouped_plan* plan, void* stream)
+{
+    if (!plan) return RMSMP_ERR_NULL;
+    if (plan->magic != kPlanMagicHost || !plan->d_table || plan->grid < 1) return RMSMP_ERR_BAD_LAYER;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    if (plan->device != device_ordinal()) return RMSMP_ERR_BAD_LAYER;
+    if (launch_stream(static_cast<const uint8_t*>(plan->d_table), plan->grid, plan->smem_bytes,
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         cudaGetLastError();
         return RMSMP_ERR_CUDA;
     }

@@ -243,6 +243,110 @@ def test_config5_grouped_launch_matches_oracle(N):
         assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
 
 
+def _grouped_case(shapes, N, layout=R.OUT_NM):
+    """Layers, device buffers, items and oracle results for a grouped launch."""
+    import torch
+    keep, items, refs = [], [], []
+    for i, (M, K) in enumerate(shapes):
+        g = synth.rng(5, 700 + i + N)
+        W = synth.weights_normal(g, (M, K))
+        ratio = synth.RATIO_SWEEP[(i + 2) % 4]
+        scheme, bits = O.assign_rows(W, ratio)
+        alpha = synth.alpha_rows(W)
+        act = synth.act_codes_uniform(g, (N, K))
+        if i % 2:
+            act = (act % 15 - 7).astype(np.int8)            # signed codes on every other layer
+        layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+        ld = (K + 15) // 16 * 16
+        a = torch.zeros((N, ld), dtype=torch.int8, device="cuda")
+        a[:, :K] = torch.from_numpy(act).cuda()
+        shape = (N, M) if layout == R.OUT_NM else (M, N)
+        y = torch.full(shape, float("nan"), dtype=torch.float32, device="cuda")
+        acc = torch.full(shape, -5, dtype=torch.int32, device="cuda") if i != 1 else None
+        step = float(np.float32(0.01 * (i + 1)))
+        keep.append((layer, d_packed, a, y, acc))
+        items.append((layer, d_packed, a, N, ld, step, y, shape[1], acc))
+        v_ref, wstep = O.quantize_rows(W, scheme, bits, alpha)
+        acc_ref = O.matmul(v_ref, act)
+        refs.append((acc_ref, _expected(acc_ref, wstep, np.float32(step))))
+    return keep, items, refs
+
+
+def _check_grouped(keep, refs, layout=R.OUT_NM):
+    for (layer, d_packed, a, y, acc), (acc_ref, y_ref) in zip(keep, refs):
+        assert R.rmsmp_last_device_status(d_packed) == R.OK
+        yh = y.cpu().numpy()
+        if layout == R.OUT_MN:
+            yh = yh.T
+        assert np.array_equal(yh.view(np.uint32), y_ref.view(np.uint32))
+        if acc is not None:
+            ah = acc.cpu().numpy()
+            assert np.array_equal(ah.T if layout == R.OUT_MN else ah, acc_ref)
+
+
+GROUPED_SHAPES = [(1024, 1024), (4096, 1024), (1024, 4096), (130, 96), (64, 40), (300, 640), (128, 128)]
+
+
+@pytest.mark.parametrize("N", [1, 8, 5, 128, 200])
+def test_config5_grouped_tensor_launch_matches_oracle(N):
+    """The grouped launch on the tensor cores (prepare once, launch): BERT-large shapes plus ragged
+    ones (row counts that are not multiples of 128, an odd number of k-blocks, K below one k-block, a
+    padded activation pitch), all four scheme ratios, signed and unsigned codes, against the oracle."""
+    import torch
+    keep, items, refs = _grouped_case(GROUPED_SHAPES, N)
+    arr = R.make_gemm_items(items)
+    table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
+    plan = R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table)
+    R.rmsmp_gemm_grouped_launch(plan)
+    torch.cuda.synchronize()
+    _check_grouped(keep, refs)
+    # the plan stays valid: new activation codes in the same buffers, second launch
+    for k, (layer, d_packed, a, y, acc) in enumerate(keep):
+        a.copy_(torch.roll(a, 1, dims=1) if a.shape[1] > 16 else a)
+        y.fill_(float("nan"))
+    R.rmsmp_gemm_grouped_launch(plan)
+    torch.cuda.synchronize()
+    for (layer, d_packed, a, y, acc) in keep:
+        assert not torch.isnan(y).any()
+
+
+def test_grouped_tensor_launch_mn_layout_and_single_layer():
+    import torch
+    keep, items, refs = _grouped_case([(384, 512), (200, 256)], 33, R.OUT_MN)
+    arr = R.make_gemm_items(items)
+    table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
+    plan = R.rmsmp_gemm_grouped_prepare(arr, R.OUT_MN, table)
+    R.rmsmp_gemm_grouped_launch(plan)
+    torch.cuda.synchronize()
+    _check_grouped(keep, refs, R.OUT_MN)
+    keep, items, refs = _grouped_case([(96, 2048)], 17)
+    arr = R.make_gemm_items(items)
+    table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
+    plan = R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table)
+    assert plan.grid == 1
+    R.rmsmp_gemm_grouped_launch(plan)
+    torch.cuda.synchronize()
+    _check_grouped(keep, refs)
+
+
+def test_grouped_tensor_launch_rejects_what_it_cannot_run():
+    import torch
+    keep, items, refs = _grouped_case([(128, 256)], 300)           # more than 256 tokens
+    arr = R.make_gemm_items(items)
+    table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table)
+    assert e.value.status == R.ERR_VARIANT
+    keep, items, refs = _grouped_case([(128, 256)], 8)
+    arr = R.make_gemm_items(items)
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table[:256])
+    assert e.value.status == R.ERR_BUFFER_TOO_SMALL
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_grouped_launch(R.rmsmp_grouped_plan())
+    assert e.value.status == R.ERR_BAD_LAYER
+
+
 # ------------------------------------------------------------------ CTA-pair kernel (long K, even row blocks, fp32 [N][M] output)
 
 @pytest.mark.parametrize("M,K,N", [
