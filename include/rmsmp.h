@@ -95,6 +95,8 @@ typedef struct rmsmp_layer {
     int32_t nP, nF4, n8;        /* rows per group */
     int32_t nblocks;            /* ceil(M/128) */
     int32_t raw_stage_bytes;    /* shared-memory bytes the packed codes of one 128-row block's k-block need (tensor kernel) */
+    int32_t max_blk[3];         /* most PoT-4 / Fixed-4 / Fixed-8 rows any one 128-row block holds (grouped kernel) */
+    int32_t reserved0;
     uint64_t off_perm, off_slot, off_wstep, off_alpha, off_kind, off_blocks, off_q4, off_q8;
     uint64_t packed_bytes;      /* size the packed buffer must have */
 } rmsmp_layer;
@@ -143,7 +145,8 @@ rmsmp_status rmsmp_quantize_pack(const float* d_W, rmsmp_w_layout w_layout,
                                  void* stream);
 
 /*
- * Parity/debug: expand a packed buffer back to integer values in ORIGINAL row order and
+ * Parity/debug (checks the level sets of Eq. 1 and Eq. 4 and the row grouping of Section 3.1 /
+ * 4.1 from outside): expand a packed buffer back to integer values in ORIGINAL row order and
  * original reduction order ([M][K], conv: [M][Cin][kh][kw]); Fixed rows give q, PoT rows
  * 0 or +-2^(e-1).  d_perm (packed -> original, M int32) and d_wstep (by original row,
  * M floats) may be NULL.  Errors: NULL, BAD_LAYER, ARCH, CUDA.
@@ -184,7 +187,9 @@ rmsmp_status rmsmp_gemm_variant(const rmsmp_layer* layer, const void* d_packed,
                                 int32_t* d_acc, rmsmp_variant variant, void* stream);
 
 /*
- * Convolution layer as an implicit GEMM (no im2col buffer): activation codes d_act are
+ * Convolution layer (Algorithm 1's forward line with filters as the weight rows: Section 3,
+ * Figure 2 -- every filter carries its own scheme and precision) as an implicit GEMM (no im2col
+ * buffer): activation codes d_act are
  * [B][H][W][Cin] (channels last), zero outside the image; output pixel index
  * n = (b*Ho + ho)*Wo + wo with Ho = (H + 2*pad - kh)/stride + 1 (same for Wo); results as in
  * rmsmp_gemm with N = B*Ho*Wo and dense leading dimension (M for NM, N for MN).
@@ -235,15 +240,15 @@ rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp
  * (Section 3.1: rows of every scheme streamed to their cores and finishing together; here all
  * layers' packed rows stream through the SMs in one kernel).  One persistent CTA per SM takes
  * blocks of 128 rows of any layer, fetches their packed codes with TMA, expands them to int8 in
- * shared memory and multiplies them with up to 256 tokens on tcgen05 (int32 accumulators in
- * tensor memory).  Results are bit for bit those of rmsmp_gemm.
+ * registers, hands them to the tensor cores through tensor memory and multiplies them with up to
+ * 128 tokens on tcgen05 (int32 accumulators in tensor memory).  Results are bit for bit those of
+ * rmsmp_gemm.
  *   rmsmp_grouped_plan_bytes    scratch size for the table of these layers on the current device.
  *   rmsmp_gemm_grouped_prepare  validates the items, builds the table (tensor maps of every
  *                               layer's packed rows and activations, work lists per SM) and queues
  *                               its upload to d_table (256-byte aligned) on `stream`; fills *plan.
- *                               Every item needs N <= 128; more tokens (up to 256) are taken while
- *                               the stages still fit shared memory, else RMSMP_ERR_VARIANT.  The call
- *                               costs host time proportional to the number of layers: do it once.
+ *                               Every item needs N <= 128, else RMSMP_ERR_VARIANT.  The call costs
+ *                               host time proportional to the number of layers: do it once.
  *   rmsmp_gemm_grouped_launch   one kernel launch from a prepared plan; may be repeated for as
  *                               long as the buffers, shapes and leading dimensions the plan was
  *                               built from stay the same (their CONTENTS may change: new weights
@@ -351,10 +356,22 @@ rmsmp_status rmsmp_gemm_builtin_scratch(const rmsmp_layer* layer, const void* d_
                                         rmsmp_out_layout out_layout, int32_t* d_acc, void* stream);
 
 /*
- * Read the device status word of a packed buffer (synchronises the stream).  Kernels never
+ * Read the device status word of a packed buffer (synchronises the stream; the paper, which
+ * describes an FPGA datapath, has no counterpart).  Kernels never
  * trap: a bounded wait that runs out stores RMSMP_ERR_TIMEOUT there and the kernel returns.
  */
 rmsmp_status rmsmp_last_device_status(const void* d_packed, void* stream);
+
+/*
+ * Self-check of the failure path (no counterpart in the paper).  Every wait inside the library's
+ * kernels is bounded: when one runs out the kernel gives up, records RMSMP_ERR_TIMEOUT in a status
+ * word and returns, so the context stays usable.  This call launches one warp that waits, with that
+ * same bounded wait, on a barrier nobody will ever signal; after `limit_cycles` SM clock cycles
+ * (1 .. 200,000,000, i.e. at most about a tenth of a second) the wait expires and the kernel stores
+ * RMSMP_ERR_TIMEOUT to *d_status_word (4 bytes of device memory, which the caller has zeroed).
+ * Asynchronous on `stream`; nothing faults, traps or hangs.  Errors: NULL, SHAPE, ARCH, CUDA.
+ */
+rmsmp_status rmsmp_selftest_bounded_wait(int64_t limit_cycles, uint32_t* d_status_word, void* stream);
 
 /*
  * Measurement helper (no counterpart in the paper): the tensor-pipe ceiling of the current GPU

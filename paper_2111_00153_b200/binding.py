@@ -32,7 +32,7 @@ EXPORTS = (
     "rmsmp_measure_mma_peak", "rmsmp_workspace_bytes", "rmsmp_expand_weights", "rmsmp_gemm_workspace",
     "rmsmp_conv_implicit_workspace", "rmsmp_gemm_builtin_scratch", "rmsmp_grouped_table_bytes",
     "rmsmp_gemm_grouped", "rmsmp_gemm_workspace_requant", "rmsmp_conv_implicit_workspace_requant",
-    "rmsmp_grouped_plan_bytes", "rmsmp_gemm_grouped_prepare", "rmsmp_gemm_grouped_launch",
+    "rmsmp_selftest_bounded_wait", "rmsmp_grouped_plan_bytes", "rmsmp_gemm_grouped_prepare", "rmsmp_gemm_grouped_launch",
 )
 
 
@@ -43,6 +43,7 @@ class rmsmp_layer(C.Structure):
         ("Cp", C.c_int32), ("Kp", C.c_int32),
         ("nP", C.c_int32), ("nF4", C.c_int32), ("n8", C.c_int32),
         ("nblocks", C.c_int32), ("raw_stage_bytes", C.c_int32),
+        ("max_blk", C.c_int32 * 3), ("reserved0", C.c_int32),
         ("off_perm", C.c_uint64), ("off_slot", C.c_uint64), ("off_wstep", C.c_uint64),
         ("off_alpha", C.c_uint64), ("off_kind", C.c_uint64), ("off_blocks", C.c_uint64),
         ("off_q4", C.c_uint64), ("off_q8", C.c_uint64),
@@ -124,6 +125,7 @@ def lib() -> C.CDLL:
                                                    C.POINTER(C.c_float), vp]
         L.rmsmp_conv_implicit_workspace_requant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
                                                             f32, f32, i32, vp, C.POINTER(C.c_float), vp]
+        L.rmsmp_selftest_bounded_wait.argtypes = [i64, vp, vp]
         L.rmsmp_measure_mma_peak.argtypes = [i32, i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
         _lib = L
     return _lib
@@ -347,6 +349,12 @@ def rmsmp_gemm_grouped_launch(plan, stream=None):
 
 def rmsmp_last_device_status(d_packed, stream=None) -> int:
     return lib().rmsmp_last_device_status(_dp(d_packed), _stream(stream))
+
+
+def rmsmp_selftest_bounded_wait(limit_cycles: int, d_status_word, stream=None):
+    """Launches the one-warp kernel whose bounded wait must run out; the status word then holds ERR_TIMEOUT."""
+    _check(lib().rmsmp_selftest_bounded_wait(limit_cycles, _dp(d_status_word), _stream(stream)),
+           "rmsmp_selftest_bounded_wait")
 
 
 def rmsmp_measure_mma_peak(d_status_word, use_bf16: bool = False, n_cols: int = 256,

@@ -38,6 +38,7 @@ struct Problem {
     const int8_t* wexp;       // [M][Kp] int8 values in original row order, or null (workspace variant)
     uint32_t* status;
     int M, Cin, kh, kw, Cp, Kp, nP, nF4, n8, nblocks, raw_stage_bytes;
+    int max_blk[3];           // most rows of each kind in any one 128-row block
     // activations: [B][H][W] pixels of `pix_pitch` bytes, Cin codes used in each
     const int8_t* act;
     int B, H, W, Ho, Wo, stride, pad;

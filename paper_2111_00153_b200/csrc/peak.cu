@@ -4,6 +4,7 @@
 // against; kind::f16 with bf16 operands (K=16) calibrates it against the known bf16 figure.
 #include <cuda.h>
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace rmsmp {
 namespace {
@@ -87,8 +88,45 @@ __global__ void __launch_bounds__(kPeakThreads, 1) mma_peak_kernel(int is_bf16, 
     }
 }
 
+// One warp waits, with the kernels' own bounded wait, on an mbarrier that nobody ever arrives on.
+// Nothing else is in flight (no bulk copy, no tensor-memory allocation), so giving up is all there is
+// to do: the wait runs out after `limit_cycles`, the abort flag goes up, the status word receives
+// RMSMP_ERR_TIMEOUT and the kernel returns normally.
+__global__ void __launch_bounds__(32, 1) wait_expiry_kernel(long long limit_cycles, uint32_t* status)
+{
+    __shared__ uint64_t s_bar;
+    __shared__ int s_abort;
+    const uint32_t bar = smem_u32(&s_bar);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    bool ok = true;
+    if (threadIdx.x == 0) ok = mbar_wait(bar, 0, &s_abort, limit_cycles);
+    ok = __all_sync(0xffffffffu, ok);
+    if (threadIdx.x == 0 && !ok && s_abort) atomicMax(status, (uint32_t)RMSMP_ERR_TIMEOUT);
+}
+
 }  // namespace
 }  // namespace rmsmp
+
+extern "C" rmsmp_status rmsmp_selftest_bounded_wait(int64_t limit_cycles, uint32_t* d_status_word, void* stream)
+{
+    using namespace rmsmp;
+    if (!d_status_word) return RMSMP_ERR_NULL;
+    if (limit_cycles < 1 || limit_cycles > 200000000LL) return RMSMP_ERR_SHAPE;      // at most ~0.1 s
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    if (major != 10) return RMSMP_ERR_ARCH;
+    wait_expiry_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>((long long)limit_cycles, d_status_word);
+    if (cudaGetLastError() != cudaSuccess) return RMSMP_ERR_CUDA;
+    return RMSMP_OK;
+}
 
 extern "C" rmsmp_status rmsmp_measure_mma_peak(int use_bf16, int n_cols, int iters, uint32_t* d_status_word, float* h_tops, float* h_ms, void* stream)
 {

@@ -36,6 +36,39 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// The same test with a suspend-time hint: the hardware may park the thread for up to `hint_ns`
+// nanoseconds (or until the phase completes) before it answers, so a waiting thread issues an
+// instruction now and then instead of spinning through the scheduler.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
+// Bounded wait built on it (same contract as mbar_wait).
+__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                 long long limit_cycles = kWaitCycles)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 16; ++i)
+            if (mbar_try_wait_parked(bar, parity, 20000u)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ bool mbar_wait_parked_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait_parked(bar, parity, abort_flag);
+    return __all_sync(0xffffffffu, ok);
+}
 // Bounded wait.  Returns false if it gave up (or another role already did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           long long limit_cycles = kWaitCycles)

@@ -506,3 +506,27 @@ def test_padded_output_rows_leave_the_padding_untouched():
         got = y.cpu().numpy()
         assert np.array_equal(got[:, :M].view(np.uint32), y_ref.reshape(N, M).view(np.uint32))
         assert (got[:, M:] == -7.0).all()
+
+
+def test_a_bounded_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """The failure path, without a fault: one warp waits on a barrier nobody signals, with the
+    kernels' own bounded wait and a limit of about a millisecond.  The status word must read
+    ERR_TIMEOUT afterwards, and an ordinary layer on the same stream must still be bit-exact."""
+    import torch
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    R.rmsmp_selftest_bounded_wait(2_000_000, status)
+    torch.cuda.synchronize()
+    assert int(status[0].item()) == R.ERR_TIMEOUT
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_selftest_bounded_wait(10 ** 10, status)          # beyond the tenth of a second the call allows
+    assert e.value.status == R.ERR_SHAPE
+    g = synth.rng(84, 1)
+    Wt = synth.weights_normal(g, (256, 512))
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    alpha = synth.alpha_rows(Wt)
+    act = synth.act_codes_uniform(g, (300, 512))
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    y, acc = Hn.gemm(layer, d_packed, act, 0.25, R.VARIANT_TENSOR)
+    _, _, acc_ref, y_ref = O.layer_linear(Wt, scheme, bits, alpha, act, np.float32(0.25))
+    assert np.array_equal(acc, acc_ref)
+    assert np.array_equal(y.view(np.uint32), y_ref.view(np.uint32))

@@ -287,7 +287,7 @@ def _check_grouped(keep, refs, layout=R.OUT_NM):
 GROUPED_SHAPES = [(1024, 1024), (4096, 1024), (1024, 4096), (130, 96), (64, 40), (300, 640), (128, 128)]
 
 
-@pytest.mark.parametrize("N", [1, 8, 5, 128, 200])
+@pytest.mark.parametrize("N", [1, 8, 5, 33, 128])
 def test_config5_grouped_tensor_launch_matches_oracle(N):
     """The grouped launch on the tensor cores (prepare once, launch): BERT-large shapes plus ragged
     ones (row counts that are not multiples of 128, an odd number of k-blocks, K below one k-block, a
@@ -331,7 +331,7 @@ def test_grouped_tensor_launch_mn_layout_and_single_layer():
 
 def test_grouped_tensor_launch_rejects_what_it_cannot_run():
     import torch
-    keep, items, refs = _grouped_case([(128, 256)], 300)           # more than 256 tokens
+    keep, items, refs = _grouped_case([(128, 256)], 129)           # more than 128 tokens
     arr = R.make_gemm_items(items)
     table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
     with pytest.raises(R.RmsmpError) as e:
