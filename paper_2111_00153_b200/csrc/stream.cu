@@ -37,7 +37,7 @@
 //                wstep * act_step, and store each lane's value to its ORIGINAL row (the 128 rows
 //                of an item are 128 adjacent outputs of a token, so the stores stay inside one
 //                512-byte window).
-// Tensor memory: columns [0, 128) and [128, 256) accumulators, [256, 512) four A stages.
+// Tensor memory: two accumulator buffers of nch * n_pad columns, then four to six A stages of 64 columns.
 // Every role looks one item ahead for the small per-item metadata (block table entry, row
 // permutation, row scales), which lives in each layer's packed buffer.
 // Every mbarrier wait is bounded; a wait that runs out sets the abort flag, all roles leave, tensor
@@ -63,11 +63,9 @@ constexpr int kExpWarps = 16;                                         // warps 8
 constexpr int kEpiWarps = 4;                                          // warps 24-27
 constexpr int kFirstMma = kProdWarps, kFirstExp = kProdWarps + kMmaWarps, kFirstEpi = kFirstExp + kExpWarps;
 constexpr int kStreamThreads = 32 * (kProdWarps + kMmaWarps + kExpWarps + kEpiWarps);      // 896
-constexpr int kAStages = 4;                                           // A stages in tensor memory
 constexpr int kAStageCols = 64;                                       // 256 codes = 64 32-bit columns per lane
-constexpr int kAccCols = 128;                                         // columns of one accumulator buffer (= max tokens)
-constexpr int kABaseCol = 2 * kAccCols;                               // first column of the A stages
-constexpr int kRingMax = 8;
+constexpr int kMaxTokens = 128;                                       // accumulator columns of one chain at most
+constexpr int kRingMax = 12;
 constexpr int kStreamSmem = 232448 - 1024;
 constexpr uint32_t kPlanMagic = 0x53545247u;                          // "STRG"
 
@@ -95,10 +93,11 @@ struct StreamItem { int32_t prob, blk; };
 struct StreamHeader {               // first 128 bytes of the table
     uint32_t magic;
     int32_t nprob, nitems, grid;
-    int32_t n_pad, nS, nch, pad_b;            // tokens rounded up to 16, ring slots, accumulator chains (1, 2 or 4)
-    uint32_t stage_bytes, b_bytes, idesc, smem_bytes;   // one ring slot: activation tiles (b_bytes) then packed codes
+    int32_t n_pad, nS, nch, nB;               // tokens rounded up to 16, slots of the packed-code ring, accumulator chains (1, 2 or 4), slots of the activation ring
+    uint32_t stage_bytes, b_bytes, idesc, smem_bytes;   // one slot of the packed-code ring / of the activation ring
+    int32_t acc_cols, nAst;                   // tensor memory: columns of one accumulator buffer (nch * n_pad); A stages behind the two buffers
     uint32_t off_first, off_items, off_probs, bytes;
-    uint32_t pad[16];
+    uint32_t pad[14];
 };
 static_assert(sizeof(StreamHeader) == 128, "header is 128 bytes");
 
@@ -230,17 +229,20 @@ stream_kernel(const uint8_t* __restrict__ table)
     const int32_t* cta_first = reinterpret_cast<const int32_t*>(table + H->off_first);
     const StreamItem* items = reinterpret_cast<const StreamItem*>(table + H->off_items);
     const StreamProblem* probs = reinterpret_cast<const StreamProblem*>(table + H->off_probs);
-    const int n_pad = H->n_pad, nS = H->nS, nch = H->nch;
+    const int n_pad = H->n_pad, nS = H->nS, nch = H->nch, nB = H->nB, nAst = H->nAst;
     const uint32_t stage_bytes = H->stage_bytes, b_bytes = H->b_bytes, idesc = H->idesc;
+    const uint32_t acc_cols = (uint32_t)H->acc_cols, a_base_col = 2u * acc_cols;
     const uint32_t b_sub = (uint32_t)n_pad * 128u;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sRing = smem_base;                     // slot s: activation tiles at + 0, packed codes at + b_bytes
+    const uint32_t sB = smem_base;                        // activation ring
+    const uint32_t sRing = sB + nB * b_bytes;             // packed-code ring
     const uint32_t sBar = sRing + nS * stage_bytes;
     const uint32_t bar_fullA = sBar, bar_emptyA = sBar + 8 * kRingMax;
     const uint32_t bar_full = sBar + 16 * kRingMax, bar_empty = sBar + 24 * kRingMax;
-    const uint32_t bar_tfull = sBar + 32 * kRingMax, bar_tempty = bar_tfull + 16;
+    const uint32_t bar_fullB = sBar + 32 * kRingMax, bar_emptyB = sBar + 40 * kRingMax;
+    const uint32_t bar_tfull = sBar + 48 * kRingMax, bar_tempty = bar_tfull + 16;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -250,8 +252,10 @@ stream_kernel(const uint8_t* __restrict__ table)
         for (int s = 0; s < kRingMax; ++s) {
             mbar_init(bar_fullA + 8 * s, kExpWarps / 2); // one arrival per expander warp of the set that has the stage
             mbar_init(bar_emptyA + 8 * s, nch);          // every issuer's tcgen05.commit
-            mbar_init(bar_full + 8 * s, kProdWarps);     // every producer warp (+ its transaction bytes)
-            mbar_init(bar_empty + 8 * s, kExpWarps / 2 + nch);   // the stage's expander warps (codes read) and every issuer's commit (activations read)
+            mbar_init(bar_full + 8 * s, kProdWarps - 1); // the three producer warps of the packed codes (+ their transaction bytes)
+            mbar_init(bar_empty + 8 * s, kExpWarps / 2); // the stage's expander warps, as soon as the codes are in their registers
+            mbar_init(bar_fullB + 8 * s, 1);             // the activation producer (+ transaction bytes)
+            mbar_init(bar_emptyB + 8 * s, nch);          // every issuer's tcgen05.commit
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_tfull + 8 * b, nch);           // every issuer's tcgen05.commit
@@ -289,13 +293,13 @@ stream_kernel(const uint8_t* __restrict__ table)
             const BlockRuns br = load_runs(P, item.blk);
             if (warp == 0) {
                 bx.tx = (uint32_t)P->hP * 128u;
-                if (lane == 0 && P->hP) { bx.map = &P->q4p; bx.row = br.p0; bx.dst = b_bytes; }
+                if (lane == 0 && P->hP) { bx.map = &P->q4p; bx.row = br.p0; bx.dst = 0u; }
             } else if (warp == 1) {
                 bx.tx = (uint32_t)P->hF * 128u;
-                if (lane == 0 && P->hF) { bx.map = &P->q4f; bx.row = P->nP + br.f0; bx.dst = b_bytes + (uint32_t)P->hP * 128u; }
+                if (lane == 0 && P->hF) { bx.map = &P->q4f; bx.row = P->nP + br.f0; bx.dst = (uint32_t)P->hP * 128u; }
             } else if (warp == 2) {
                 bx.tx = 2u * (uint32_t)P->hE * 128u;
-                if (lane < 2 && P->hE) { bx.map = &P->q8; bx.row = br.e0; bx.dst = b_bytes + (uint32_t)(P->hP + P->hF + lane * P->hE) * 128u; }
+                if (lane < 2 && P->hE) { bx.map = &P->q8; bx.row = br.e0; bx.dst = (uint32_t)(P->hP + P->hF + lane * P->hE) * 128u; }
             } else {
                 bx.tx = b_sub;                            // per k-block
                 if (lane < 2) { bx.map = &P->act; bx.row = 0; bx.dst = (uint32_t)lane * b_sub; }
@@ -314,17 +318,21 @@ stream_kernel(const uint8_t* __restrict__ table)
             }
             const Box nxt = box_of(it + 1);               // in flight while this item streams
             const int nkb = P->nkb, npairs = (nkb + 1) >> 1;
+            // warps 0-2 fill the packed-code ring, warp 3 the activation ring (its own depth and barriers)
+            const uint32_t ring_n = (warp == 3) ? (uint32_t)nB : (uint32_t)nS;
+            const uint32_t bar_e = (warp == 3) ? bar_emptyB : bar_empty, bar_f = (warp == 3) ? bar_fullB : bar_full;
+            const uint32_t ring0 = (warp == 3) ? sB : sRing, ring_b = (warp == 3) ? b_bytes : stage_bytes;
             for (int kp = 0; kp < npairs; ++kp) {
-                if (!mbar_wait_parked_warp(bar_empty + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
-                const uint32_t fbar = bar_full + 8 * sr;
+                if (!mbar_wait_parked_warp(bar_e + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
+                const uint32_t fbar = bar_f + 8 * sr;
                 const bool two = 2 * kp + 1 < nkb;
                 if (lane == 0) mbar_arrive_expect_tx(fbar, (warp == 3 && two) ? 2u * cur.tx : cur.tx);
                 __syncwarp();
                 // byte offset into the source row: 4-bit runs 128 bytes per stage; 8-bit runs and activations 128 per k-block
                 const int x = (warp < 2) ? kp * 128 : (2 * kp + lane) * 128;
                 if (cur.map && !(warp == 3 && lane == 1 && !two))
-                    tma_load_2d(sRing + sr * stage_bytes + cur.dst, cur.map, fbar, x, cur.row);
-                if (++sr == (uint32_t)nS) { sr = 0; phR ^= 1; }
+                    tma_load_2d(ring0 + sr * ring_b + cur.dst, cur.map, fbar, x, cur.row);
+                if (++sr == ring_n) { sr = 0; phR ^= 1; }
             }
             cur = nxt;
         }
@@ -337,7 +345,7 @@ stream_kernel(const uint8_t* __restrict__ table)
         if (me < nch) {
             const bool issuer = (lane == 0);
             uint32_t sa = 0, phA = 0, sb = 0, phB = 0, n = 0;
-            const uint64_t desc_b0 = smem_desc_kmajor(sRing, 128);
+            const uint64_t desc_b0 = smem_desc_kmajor(sB, 128);
             const uint32_t b_lo0 = (uint32_t)desc_b0, desc_hi = (uint32_t)(desc_b0 >> 32);
             bool ok = true;
             for (int it = it0; it < it1 && ok && !*abort_flag; ++it, ++n) {
@@ -348,11 +356,11 @@ stream_kernel(const uint8_t* __restrict__ table)
                 const uint32_t ab = n & 1;
                 if (!mbar_wait_parked(bar_tempty + 8 * ab, ((n >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + ab * kAccCols + (uint32_t)(me * n_pad);
+                const uint32_t d_tmem = tmem_base + ab * acc_cols + (uint32_t)(me * n_pad);
                 for (int kp = 0; kp < npairs; ++kp) {
-                    if (!mbar_wait_parked(bar_full + 8 * sb, phB, abort_flag) || !mbar_wait_parked(bar_fullA + 8 * sa, phA, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_parked(bar_fullB + 8 * sb, phB, abort_flag) || !mbar_wait_parked(bar_fullA + 8 * sa, phA, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_t = tmem_base + kABaseCol + sa * kAStageCols, b_lo = b_lo0 + sb * (stage_bytes >> 4);
+                    const uint32_t a_t = tmem_base + a_base_col + sa * kAStageCols, b_lo = b_lo0 + sb * (b_bytes >> 4);
                     if (issuer) {
                         // a 32-code step is 8 columns of A and 32 bytes (two 16-byte units) of a B row; this
                         // issuer's first instruction of the item overwrites its chain
@@ -362,10 +370,10 @@ stream_kernel(const uint8_t* __restrict__ table)
                             mma_i8_tmem_a(d_tmem, a_t + 8 * j, b_j, desc_hi, idesc, (kp == 0 && j == me) ? 0u : 1u);
                         }
                         mma_commit(bar_emptyA + 8 * sa);
-                        mma_commit(bar_empty + 8 * sb);
+                        mma_commit(bar_emptyB + 8 * sb);
                     }
-                    if (++sa == (uint32_t)kAStages) { sa = 0; phA ^= 1; }
-                    if (++sb == (uint32_t)nS) { sb = 0; phB ^= 1; }
+                    if (++sa == (uint32_t)nAst) { sa = 0; phA ^= 1; }
+                    if (++sb == (uint32_t)nB) { sb = 0; phB ^= 1; }
                 }
                 if (!ok) break;
                 if (issuer) mma_commit(bar_tfull + 8 * ab);
@@ -380,8 +388,9 @@ stream_kernel(const uint8_t* __restrict__ table)
         const int set = ((warp - kFirstExp) >> 2) & 1;   // which stages: those with (stage index & 1) == set
         const int half = (warp - kFirstExp) >> 3;        // which k-block of a stage: its 32-code steps 4 * half .. + 3
         const int slot = quarter * 32 + lane;            // the thread's row of every item, in packed order
-        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + kABaseCol + 32 * half;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + a_base_col + 32 * half;
         uint32_t t = 0;                                  // stages this CTA has been through
+        uint32_t sr = 0, phR = 0, sa = 0, phA = 0;       // ring positions of stage t (advanced for every stage, taken or not)
         auto meta_of = [&](int it) -> uint32_t {
             if (it >= it1) return 3u << 30;
             const StreamItem item = items[it];
@@ -396,24 +405,25 @@ stream_kernel(const uint8_t* __restrict__ table)
             const int npairs = (P->nkb + 1) >> 1;
             const uint32_t nxt = meta_of(it + 1);         // in flight during this item
             for (int kp = 0; kp < npairs; ++kp, ++t) {
-                if ((int)(t & 1u) != set) continue;
-                const uint32_t sr = t % (uint32_t)nS, phR = (t / (uint32_t)nS) & 1u;
-                const uint32_t sa = t % (uint32_t)kAStages, phA = (t / (uint32_t)kAStages) & 1u;
-                if (!mbar_wait_parked_warp(bar_full + 8 * sr, phR, abort_flag)) { ok = false; break; }
-                const uint32_t raw = sRing + sr * stage_bytes + b_bytes;
-                uint32_t w[16];
-                stream_expand(cur, raw, 2 * half, w);
-                if (!mbar_wait_parked_warp(bar_emptyA + 8 * sa, phA ^ 1, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                tmem_st16(t_lane + sa * kAStageCols, w);
-                stream_expand(cur, raw, 2 * half + 1, w);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_empty + 8 * sr);           // the raw bytes are in registers
-                tmem_st16(t_lane + sa * kAStageCols + 16, w);
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_fullA + 8 * sa);
+                if ((int)(t & 1u) == set) {
+                    if (!mbar_wait_parked_warp(bar_full + 8 * sr, phR, abort_flag)) { ok = false; break; }
+                    const uint32_t raw = sRing + sr * stage_bytes;
+                    uint32_t w[16];
+                    stream_expand(cur, raw, 2 * half, w);
+                    if (!mbar_wait_parked_warp(bar_emptyA + 8 * sa, phA ^ 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    tmem_st16(t_lane + sa * kAStageCols, w);
+                    stream_expand(cur, raw, 2 * half + 1, w);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_empty + 8 * sr);       // the raw bytes are in registers: the slot can be refilled
+                    tmem_st16(t_lane + sa * kAStageCols + 16, w);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_fullA + 8 * sa);
+                }
+                if (++sr == (uint32_t)nS) { sr = 0; phR ^= 1; }
+                if (++sa == (uint32_t)nAst) { sa = 0; phA ^= 1; }
             }
             cur = nxt;
         }
@@ -446,7 +456,7 @@ stream_kernel(const uint8_t* __restrict__ table)
             const uint32_t ab = n & 1;
             if (!mbar_wait_parked_warp(bar_tfull + 8 * ab, (n >> 1) & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * kAccCols;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * acc_cols;
             const int N = P->N;
             float* const out = P->out;
             int32_t* const acc = P->acc;
@@ -529,7 +539,7 @@ size_t stream_table_bytes(int count, int64_t nitems, int sms)
 // Can this problem be part of a grouped tensor-core launch?
 bool stream_supported(const Problem& p)
 {
-    if (p.kh != 1 || p.kw != 1 || p.N < 1 || p.N > kAccCols) return false;
+    if (p.kh != 1 || p.kw != 1 || p.N < 1 || p.N > kMaxTokens) return false;
     if (p.pix_pitch % 16 != 0 || (reinterpret_cast<uintptr_t>(p.act) & 15) != 0) return false;
     if (p.max_blk[0] + p.max_blk[1] + p.max_blk[2] <= 0) return false;      // descriptor from an older rmsmp_layer_init
     return tensor_map_encoder() != nullptr;
@@ -563,14 +573,19 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
     // consecutive MMAs into one accumulator wait for each other; with few tokens the accumulator buffer has room
     // for several chains that the 32-code steps take in turn (summed in the epilogue)
     H->nch = H->n_pad <= 32 ? 4 : (H->n_pad <= 64 ? 2 : 1);
+    H->acc_cols = H->nch * H->n_pad;                              // <= 128
+    H->nAst = std::min(6, (512 - 2 * H->acc_cols) / kAStageCols) & ~1;      // even: the two expander sets alternate
     H->b_bytes = (uint32_t)(2 * H->n_pad * 128);
-    H->stage_bytes = H->b_bytes + (uint32_t)raw_rows * 128u;      // multiples of 1024: every box starts on a swizzle atom
-    // the ring takes all of shared memory: its depth is what is in flight from HBM (the expanded weights
-    // live in tensor memory)
+    H->stage_bytes = (uint32_t)raw_rows * 128u;                   // multiples of 1024: every box starts on a swizzle atom
+    // Shared memory: a packed-code slot is held from the moment its copy is started until the expanders have the
+    // bytes in registers, i.e. for one trip to HBM, so the number of such slots is what is in flight from HBM; an
+    // activation slot is held until its MMAs have finished.  Activations get up to six slots (a quarter of the
+    // memory at most), the packed codes everything else.
     const int64_t avail = kStreamSmem - 1024 - 64 * kRingMax;
-    H->nS = (int)std::min<int64_t>(kRingMax, avail / H->stage_bytes);
+    H->nB = (int)std::min<int64_t>(6, std::max<int64_t>(2, avail / 4 / H->b_bytes));
+    H->nS = (int)std::min<int64_t>(kRingMax, (avail - (int64_t)H->nB * H->b_bytes) / H->stage_bytes);
     if (H->nS < 2) return false;
-    H->smem_bytes = (uint32_t)(H->nS * H->stage_bytes + 1024 + 64 * kRingMax);
+    H->smem_bytes = (uint32_t)(H->nB * H->b_bytes + H->nS * H->stage_bytes + 1024 + 64 * kRingMax);
     // kind::i8: int32 accumulate, signed 8-bit A and B, both K-major, N/8 at bit 17, M/16 at bit 24
     H->idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(H->n_pad >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
     H->off_first = (uint32_t)L.off_first; H->off_items = (uint32_t)L.off_items; H->off_probs = (uint32_t)L.off_probs;
