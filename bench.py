@@ -412,6 +412,7 @@ def run_ours(args):
                              "peak_source": "tcgen05.mma kind::i8 M=128 N=256 loop measured in this run (rmsmp_measure_mma_peak); "
                                             "2 x measured bf16 GEMM = %.0f" % (2 * peaks["bf16_tflops"]),
                              "layers": len(tb)} if tb and i8_peak > 0 else None),
+        "roofline_weights": (weights_leg(R, torch, peaks) if (world == 1 and not args.no_weights_leg) else None),
         "roofline_per_layer": binding_roof_summary(H, conv_ms_layer, alg, batch, peaks["hbm_gbs"], i8_peak, peaks),
         "per_layer": [{"name": h["L"].name, "M": h["L"].M, "K": h["L"].K, "N": d["N"], "ms": float(ms),
                        "tops": layer_ops(h["L"], batch) / (ms * 1e-3) / 1e12, "gbs": float(a / (ms * 1e-3) / 1e9)}
@@ -422,6 +423,69 @@ def run_ours(args):
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def bert_large_stack(R, torch, ratio=RATIO, layers=24):
+    """Config 5 as one cold stream: the linears of `layers` BERT-large encoder layers (4 x 1024x1024, 4096x1024,
+    1024x4096 each), seeded N(0, 0.02) weights, rows assigned by variance rank, packed on the device."""
+    out = []
+    for l in range(layers):
+        for j, (M, K) in enumerate(((1024, 1024),) * 4 + ((4096, 1024), (1024, 4096))):
+            W = synth.weights_normal(synth.rng(5, 100 * l + j), (M, K))
+            scheme, bits = R.rmsmp_assign_rows(W, ratio)
+            lay = R.rmsmp_layer_init(M, K, 1, 1, scheme, bits)
+            pk = torch.empty(lay.packed_bytes, dtype=torch.uint8, device="cuda")
+            R.rmsmp_quantize_pack(torch.from_numpy(W).cuda(), R.W_LINEAR, lay, scheme, bits, synth.alpha_rows(W), R.POT_NEAREST, pk)
+            out.append((lay, pk))
+    torch.cuda.synchronize()
+    return out
+
+
+def weights_leg(R, torch, peaks, tokens=(1, 8, 128), reps=5, launches=20):
+    """The weight-bound regime (config 5): the whole BERT-large stack (144 linears, ~160 MB of packed codes,
+    more than L2) through ONE grouped tensor-core launch per pass, at a few token counts.  The plan is
+    prepared once; a pass is one launch; `launches` passes run back to back between two events."""
+    stack = bert_large_stack(R, torch)
+    rows = []
+    for N in tokens:
+        keep, items, alg, wbytes, ops = [], [], 0, 0, 0
+        g = synth.rng(5, 9000 + N)
+        for lay, pk in stack:
+            M, K = lay.M, lay.Cin
+            act = torch.from_numpy(synth.act_codes_uniform(g, (N, K))).cuda()
+            y = torch.empty((N, M), dtype=torch.float32, device="cuda")
+            keep.append((act, y))
+            items.append((lay, pk, act, N, K, 0.1, y, M, None))
+            w = (lay.nP + lay.nF4) * K // 2 + lay.n8 * K + 8 * M
+            wbytes += w
+            alg += w + N * K + 4 * N * M
+            ops += 2 * M * K * N
+        arr = R.make_gemm_items(items)
+        table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
+        plan = R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table)
+        for _ in range(50):
+            R.rmsmp_gemm_grouped_launch(plan)
+        torch.cuda.synchronize()
+        best = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(launches):
+                R.rmsmp_gemm_grouped_launch(plan)
+            b.record()
+            torch.cuda.synchronize()
+            best.append(a.elapsed_time(b) / launches)
+        ms = float(np.median(best))
+        for lay, pk in stack[:3]:
+            assert R.rmsmp_last_device_status(pk) == R.OK
+        rows.append({"tokens": N, "us": ms * 1e3, "gbs": alg / (ms * 1e-3) / 1e9, "frac": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "tops": ops / (ms * 1e-3) / 1e12, "algorithmic_bytes": float(alg), "packed_weight_bytes": float(wbytes)})
+        del keep, items, arr, table, plan
+    head = rows[min(1, len(rows) - 1)]                    # the N = 8 row speaks for the regime
+    return {"bound": "hbm", "kernel": "stream_kernel (rmsmp_gemm_grouped_launch: 144 BERT-large linears in one launch, ratio %d:%d:%d)" % RATIO,
+            "achieved": head["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": head["frac"], "traffic": None,
+            "at_tokens": head["tokens"], "rows": rows,
+            "timing": "%d launches back to back between two events, median of %d; the packed weights (160 MB) exceed L2" % (launches, reps)}
 
 
 def binding_roof_summary(H, ms_layer, alg_bytes, batch, hbm_gbs, i8_peak, peaks):
@@ -673,6 +737,14 @@ def run_suite(args):
                     ratio=ratio, pool=24, only=("simt_dp4a", "shift_add"), iters=48)
     # config 5 as the natural cold stream: the whole BERT-large stack (24 x six linears, ~158 MB of
     # packed weights, larger than L2) in ONE grouped launch; the table upload is part of the call.
+    if want("grouped"):
+        leg = weights_leg(R, torch, peaks)
+        for r in leg["rows"]:
+            rec = {"suite": "config5", "shape": "bert-large stack, 144 linears, N=%d, one grouped launch (plan prepared once)" % r["tokens"],
+                   "N": r["tokens"], "ratio": list(RATIO), "variant": "grouped_tensor", "us": r["us"], "tops": r["tops"], "gbs": r["gbs"],
+                   "frac_int8_peak": r["tops"] / i8_peak, "frac_hbm": r["frac"], "weights": "cold stream"}
+            rows.append(rec)
+            print(json.dumps(rec))
     for N in (1, 8):
         if not want("grouped"):
             break
@@ -712,6 +784,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-batch", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-weights-leg", action="store_true",
+                    help="skip the weight-bound leg (the grouped BERT-large launch reported as roofline_weights)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--variant", default="workspace", choices=["workspace", "smem"],
                     help="tensor-core path: expand the weight codes once into scratch memory (default) "

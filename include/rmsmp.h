@@ -95,8 +95,6 @@ typedef struct rmsmp_layer {
     int32_t nP, nF4, n8;        /* rows per group */
     int32_t nblocks;            /* ceil(M/128) */
     int32_t raw_stage_bytes;    /* shared-memory bytes the packed codes of one 128-row block's k-block need (tensor kernel) */
-    int32_t max_blk[3];         /* most PoT-4 / Fixed-4 / Fixed-8 rows any one 128-row block holds (grouped kernel) */
-    int32_t reserved0;
     uint64_t off_perm, off_slot, off_wstep, off_alpha, off_kind, off_blocks, off_q4, off_q8;
     uint64_t packed_bytes;      /* size the packed buffer must have */
 } rmsmp_layer;

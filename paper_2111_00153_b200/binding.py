@@ -43,7 +43,6 @@ class rmsmp_layer(C.Structure):
         ("Cp", C.c_int32), ("Kp", C.c_int32),
         ("nP", C.c_int32), ("nF4", C.c_int32), ("n8", C.c_int32),
         ("nblocks", C.c_int32), ("raw_stage_bytes", C.c_int32),
-        ("max_blk", C.c_int32 * 3), ("reserved0", C.c_int32),
         ("off_perm", C.c_uint64), ("off_slot", C.c_uint64), ("off_wstep", C.c_uint64),
         ("off_alpha", C.c_uint64), ("off_kind", C.c_uint64), ("off_blocks", C.c_uint64),
         ("off_q4", C.c_uint64), ("off_q8", C.c_uint64),

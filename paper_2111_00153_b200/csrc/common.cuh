@@ -38,7 +38,6 @@ struct Problem {
     const int8_t* wexp;       // [M][Kp] int8 values in original row order, or null (workspace variant)
     uint32_t* status;
     int M, Cin, kh, kw, Cp, Kp, nP, nF4, n8, nblocks, raw_stage_bytes;
-    int max_blk[3];           // most rows of each kind in any one 128-row block
     // activations: [B][H][W] pixels of `pix_pitch` bytes, Cin codes used in each
     const int8_t* act;
     int B, H, W, Ho, Wo, stride, pad;
@@ -102,6 +101,7 @@ int grouped_fill_table(const Problem* probs, int count, uint8_t* h_table);
 cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t total, int nt, cudaStream_t st);
 // grouped tensor-core launch (stream.cu): table size, per-problem support test, host-side table and
 // launch geometry, launch
+int64_t stream_items_of(int nP, int nF4, int n8);
 size_t stream_table_bytes(int count, int64_t nitems, int sms);
 bool stream_supported(const Problem& p);
 bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_table, size_t table_bytes,

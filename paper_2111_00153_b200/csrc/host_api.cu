@@ -124,7 +124,6 @@ void fill_problem(Problem& p, const rmsmp_layer* L, const void* d_packed)
     p.M = L->M; p.Cin = L->Cin; p.kh = L->kh; p.kw = L->kw; p.Cp = L->Cp; p.Kp = L->Kp;
     p.nP = L->nP; p.nF4 = L->nF4; p.n8 = L->n8; p.nblocks = L->nblocks;
     p.raw_stage_bytes = L->raw_stage_bytes;
-    for (int k = 0; k < 3; ++k) p.max_blk[k] = L->max_blk[k];
     p.wexp = nullptr;
     p.rq_codes = nullptr; p.rq_alpha = 1.0f; p.rq_kind = 0; p.ld_codes = 0;
 }
@@ -270,7 +269,6 @@ rmsmp_status rmsmp_layer_init(rmsmp_layer* L, int M, int Cin, int kh, int kw,
         for (int r = b0; r < M && r < b0 + kBlockRows; ++r) ++c[row_kind(h_scheme[r], h_bits[r])];
         const int bytes = ((c[0] + 15) / 16 * 16 + (c[1] + 15) / 16 * 16) * 64 + (c[2] + 15) / 16 * 16 * 128;
         raw_max = std::max(raw_max, bytes);
-        for (int k = 0; k < 3; ++k) L->max_blk[k] = std::max(L->max_blk[k], c[k]);
     }
     L->raw_stage_bytes = raw_max;
     uint64_t off = 256;
@@ -519,7 +517,8 @@ rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp
 static int64_t grouped_row_blocks(const rmsmp_gemm_item* h_items, int count)
 {
     int64_t n = 0;
-    for (int i = 0; i < count; ++i) n += h_items[i].layer ? h_items[i].layer->nblocks : 0;
+    for (int i = 0; i < count; ++i)
+        if (h_items[i].layer) n += stream_items_of(h_items[i].layer->nP, h_items[i].layer->nF4, h_items[i].layer->n8);
     return n;
 }
 

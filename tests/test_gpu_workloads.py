@@ -323,7 +323,7 @@ def test_grouped_tensor_launch_mn_layout_and_single_layer():
     arr = R.make_gemm_items(items)
     table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
     plan = R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table)
-    assert plan.grid == 1
+    assert plan.grid == 3                      # one tile per kind
     R.rmsmp_gemm_grouped_launch(plan)
     torch.cuda.synchronize()
     _check_grouped(keep, refs)
