@@ -413,6 +413,7 @@ def run_ours(args):
                                             "2 x measured bf16 GEMM = %.0f" % (2 * peaks["bf16_tflops"]),
                              "layers": len(tb)} if tb and i8_peak > 0 else None),
         "roofline_weights": (weights_leg(R, torch, peaks) if (world == 1 and not args.no_weights_leg) else None),
+        "per_config": (configs_leg(R, torch, peaks, i8_peak) if (world == 1 and not args.no_weights_leg and i8_peak > 0) else None),
         "roofline_per_layer": binding_roof_summary(H, conv_ms_layer, alg, batch, peaks["hbm_gbs"], i8_peak, peaks),
         "per_layer": [{"name": h["L"].name, "M": h["L"].M, "K": h["L"].K, "N": d["N"], "ms": float(ms),
                        "tops": layer_ops(h["L"], batch) / (ms * 1e-3) / 1e12, "gbs": float(a / (ms * 1e-3) / 1e9)}
@@ -439,6 +440,58 @@ def bert_large_stack(R, torch, ratio=RATIO, layers=24):
             out.append((lay, pk))
     torch.cuda.synchronize()
     return out
+
+
+def configs_leg(R, torch, peaks, i8_peak):
+    """Throughput of the other workload configurations (1: one small linear layer; 2: the 256->256 3x3
+    convolution at 14x14, batch 32; 3: the four BERT-base linears at 4096 tokens), each through the
+    call the benchmark's stack uses (weights expanded once into scratch, tensor cores), replayed 20
+    times between two events.  Algorithmic bytes and ops as for the stack; every shape is reported
+    against both roofs and names the one that binds it."""
+    rows = []
+
+    def one(cfg, name, M, Cin, k, stride, pad, B, H, kind):
+        conv = k > 1 or H > 1
+        g = synth.rng(6, M + Cin + k + B)
+        W = synth.weights_kaiming(g, M, Cin, k, k) if conv else synth.weights_normal(g, (M, Cin)).reshape(M, Cin, 1, 1)
+        scheme, bits = R.rmsmp_assign_rows(W, RATIO)
+        lay = R.rmsmp_layer_init(M, Cin, k, k, scheme, bits)
+        pk = torch.empty(lay.packed_bytes, dtype=torch.uint8, device="cuda")
+        R.rmsmp_quantize_pack(torch.from_numpy(W).cuda(), R.W_CONV_OIHW, lay, scheme, bits, synth.alpha_rows(W), R.POT_NEAREST, pk)
+        ws = torch.empty(R.rmsmp_workspace_bytes(lay), dtype=torch.int8, device="cuda")
+        R.rmsmp_expand_weights(lay, pk, ws)
+        Ho = (H + 2 * pad - k) // stride + 1
+        N = B * Ho * Ho
+        lo, hi = (0, 16) if kind == R.ACT_U4 else (-7, 8)
+        act = torch.randint(lo, hi, (B, H, H, Cin), dtype=torch.int8, device="cuda")
+        y = torch.empty((N, M), dtype=torch.float32, device="cuda")
+        fn = lambda: R.rmsmp_conv_implicit_workspace(lay, pk, ws, act, B, H, H, stride, pad, 0.1, y, R.OUT_NM, None)
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(20):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) / 20)
+        ms = float(np.median(ts))
+        ops = 2 * M * Cin * k * k * N
+        alg = (lay.nP + lay.nF4) * lay.K // 2 + lay.n8 * lay.K + 8 * M + B * H * H * Cin + 4 * N * M
+        t_h, t_t = alg / (peaks["hbm_gbs"] * 1e9) * 1e3, ops / (i8_peak * 1e12) * 1e3
+        rows.append({"config": cfg, "shape": name, "M": M, "K": Cin * k * k, "N": N, "us": ms * 1e3, "tops": ops / (ms * 1e-3) / 1e12,
+                     "gbs": alg / (ms * 1e-3) / 1e9, "bound": "tensor" if t_t > t_h else "hbm", "frac": max(t_h, t_t) / ms,
+                     "weights": "L2-resident replay"})
+
+    one(1, "linear 256x512, 64 tokens", 256, 512, 1, 1, 0, 64, 1, R.ACT_U4)
+    L = synth.CONFIG2_CONV
+    one(2, "conv 256->256 3x3 on 14x14, batch 32", L.M, L.Cin, 3, 1, 1, 32, 14, R.ACT_U4)
+    for nm, M, K in synth.BERT_BASE_LINEARS:
+        one(3, "bert-base %s %dx%d, 4096 tokens" % (nm, M, K), M, K, 1, 1, 0, 4096, 1, R.ACT_S4)
+    return rows
 
 
 def weights_leg(R, torch, peaks, tokens=(1, 8, 128), reps=5, launches=20):

@@ -143,6 +143,32 @@ rmsmp_status rmsmp_quantize_pack(const float* d_W, rmsmp_w_layout w_layout,
                                  void* stream);
 
 /*
+ * The same from the ratio alone: the row assignment runs on the device (Section 3.1: of two rows
+ * the one with the lower variance takes PoT; Section 3.3: ratio PoT-4 : Fixed-4 : Fixed-8 = A : B : C;
+ * Algorithm 1's assignment block, with the variance rank standing in for its Hessian ranking as in
+ * rmsmp_assign_rows), so nothing about the weights has to be known on the host.
+ *   rmsmp_layer_init_ratio       describes the layer from the ratio: the row counts per kind follow
+ *                                from M and A:B:C (n8 = floor(M*C/100 + 1/2), nP = floor(M*A/100 + 1/2),
+ *                                the rest Fixed-4), which fixes the packed layout.  Host only.  M <= 65536.
+ *   rmsmp_assign_scratch_bytes   device scratch the assignment needs (16 bytes per row).
+ *   rmsmp_assign_quantize_pack   per-row population variance (double, two passes in reduction order),
+ *                                rank by (variance, row index), kinds from the rank, stable grouping,
+ *                                all metadata of the packed buffer, then the quantizers of
+ *                                rmsmp_quantize_pack.  d_alpha: M clip values on the device, or NULL for
+ *                                alpha_r = max |w| of the row (1 for an all-zero row).  d_scheme / d_bits
+ *                                (optional, M bytes each on the device) receive the assignment.  The
+ *                                result equals rmsmp_assign_rows + rmsmp_quantize_pack bit for bit.
+ * Errors: NULL, BAD_LAYER, SHAPE, SCHEME (descriptor built for another ratio), BUFFER_TOO_SMALL, ALIGN,
+ * ARCH, CUDA.
+ */
+rmsmp_status rmsmp_layer_init_ratio(rmsmp_layer* layer, int M, int Cin, int kh, int kw, int A, int B, int C);
+rmsmp_status rmsmp_assign_scratch_bytes(int M, size_t* bytes);
+rmsmp_status rmsmp_assign_quantize_pack(const float* d_W, rmsmp_w_layout w_layout, const rmsmp_layer* layer,
+                                        int A, int B, int C, const float* d_alpha, rmsmp_pot_mode pot_mode,
+                                        void* d_packed, size_t packed_bytes, void* d_scratch, size_t scratch_bytes,
+                                        uint8_t* d_scheme, uint8_t* d_bits, void* stream);
+
+/*
  * Parity/debug (checks the level sets of Eq. 1 and Eq. 4 and the row grouping of Section 3.1 /
  * 4.1 from outside): expand a packed buffer back to integer values in ORIGINAL row order and
  * original reduction order ([M][K], conv: [M][Cin][kh][kw]); Fixed rows give q, PoT rows

@@ -32,7 +32,7 @@ EXPORTS = (
     "rmsmp_measure_mma_peak", "rmsmp_workspace_bytes", "rmsmp_expand_weights", "rmsmp_gemm_workspace",
     "rmsmp_conv_implicit_workspace", "rmsmp_gemm_builtin_scratch", "rmsmp_grouped_table_bytes",
     "rmsmp_gemm_grouped", "rmsmp_gemm_workspace_requant", "rmsmp_conv_implicit_workspace_requant",
-    "rmsmp_selftest_bounded_wait", "rmsmp_grouped_plan_bytes", "rmsmp_gemm_grouped_prepare", "rmsmp_gemm_grouped_launch",
+    "rmsmp_layer_init_ratio", "rmsmp_assign_scratch_bytes", "rmsmp_assign_quantize_pack", "rmsmp_selftest_bounded_wait", "rmsmp_grouped_plan_bytes", "rmsmp_gemm_grouped_prepare", "rmsmp_gemm_grouped_launch",
 )
 
 
@@ -124,6 +124,10 @@ def lib() -> C.CDLL:
                                                    C.POINTER(C.c_float), vp]
         L.rmsmp_conv_implicit_workspace_requant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
                                                             f32, f32, i32, vp, C.POINTER(C.c_float), vp]
+        L.rmsmp_layer_init_ratio.argtypes = [C.POINTER(rmsmp_layer), i32, i32, i32, i32, i32, i32, i32]
+        L.rmsmp_assign_scratch_bytes.argtypes = [i32, C.POINTER(C.c_size_t)]
+        L.rmsmp_assign_quantize_pack.argtypes = [vp, i32, C.POINTER(rmsmp_layer), i32, i32, i32, vp, i32, vp, C.c_size_t,
+                                                 vp, C.c_size_t, vp, vp, vp]
         L.rmsmp_selftest_bounded_wait.argtypes = [i64, vp, vp]
         L.rmsmp_measure_mma_peak.argtypes = [i32, i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
         _lib = L
@@ -348,6 +352,28 @@ def rmsmp_gemm_grouped_launch(plan, stream=None):
 
 def rmsmp_last_device_status(d_packed, stream=None) -> int:
     return lib().rmsmp_last_device_status(_dp(d_packed), _stream(stream))
+
+
+def rmsmp_layer_init_ratio(M: int, Cin: int, kh: int, kw: int, ratio) -> rmsmp_layer:
+    layer = rmsmp_layer()
+    _check(lib().rmsmp_layer_init_ratio(C.byref(layer), M, Cin, kh, kw, int(ratio[0]), int(ratio[1]), int(ratio[2])),
+           "rmsmp_layer_init_ratio")
+    return layer
+
+
+def rmsmp_assign_scratch_bytes(M: int) -> int:
+    n = C.c_size_t(0)
+    _check(lib().rmsmp_assign_scratch_bytes(M, C.byref(n)), "rmsmp_assign_scratch_bytes")
+    return n.value
+
+
+def rmsmp_assign_quantize_pack(d_W, w_layout: int, layer, ratio, d_alpha, pot_mode: int, d_packed, d_scratch,
+                               d_scheme=None, d_bits=None, stream=None):
+    """Row assignment on the device + quantize + pack, from the ratio alone."""
+    _check(lib().rmsmp_assign_quantize_pack(_dp(d_W), w_layout, C.byref(layer), int(ratio[0]), int(ratio[1]), int(ratio[2]),
+                                            _dp(d_alpha), pot_mode, _dp(d_packed), d_packed.numel() * d_packed.element_size(),
+                                            _dp(d_scratch), d_scratch.numel() * d_scratch.element_size(), _dp(d_scheme),
+                                            _dp(d_bits), _stream(stream)), "rmsmp_assign_quantize_pack")
 
 
 def rmsmp_selftest_bounded_wait(limit_cycles: int, d_status_word, stream=None):

@@ -87,6 +87,10 @@ rmsmp_status dispatch_problem(Problem& p, rmsmp_variant variant, cudaStream_t st
 // kernels (each returns the CUDA launch error, cudaSuccess if fine)
 cudaError_t launch_pack(const float* dW, int conv_oihw, const rmsmp_layer& L, int pot_mode,
                         uint8_t* blob, cudaStream_t st);
+// row assignment on the device + the packed buffer's metadata (assign.cu); scratch of assign_scratch_bytes(M)
+size_t assign_scratch_bytes(int M);
+cudaError_t launch_assign_meta(const float* dW, const rmsmp_layer& L, const float* d_alpha, int pot_mode, uint8_t* blob,
+                               void* d_scratch, uint8_t* d_scheme, uint8_t* d_bits, cudaStream_t st);
 // copies `bytes` from mapped pinned host memory (device view, 16-byte aligned) to device memory
 cudaError_t launch_fetch_mapped(void* d_dst, const void* mapped_src, size_t bytes, cudaStream_t st);
 cudaError_t launch_unpack(const rmsmp_layer& L, const uint8_t* blob, int8_t* values,

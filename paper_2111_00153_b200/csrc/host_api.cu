@@ -241,19 +241,12 @@ rmsmp_status rmsmp_assign_rows(const float* h_W, int M, int K, int A, int B, int
     return RMSMP_OK;
 }
 
-rmsmp_status rmsmp_layer_init(rmsmp_layer* L, int M, int Cin, int kh, int kw,
-                              const uint8_t* h_scheme, const uint8_t* h_bits)
+// Shape checks, padded sizes and section offsets of a layer with cnt[] rows per kind.
+static rmsmp_status layer_layout(rmsmp_layer* L, int M, int Cin, int kh, int kw, const int cnt[3])
 {
-    if (!L || !h_scheme || !h_bits) return RMSMP_ERR_NULL;
     if (M < 1 || M > (1 << 20) || Cin < 1 || kh < 1 || kw < 1 || kh > 16 || kw > 16)
         return RMSMP_ERR_SHAPE;
     if ((int64_t)Cin * kh * kw > 1000000) return RMSMP_ERR_SHAPE;
-    int cnt[3] = {0, 0, 0};
-    for (int r = 0; r < M; ++r) {
-        const int k = row_kind(h_scheme[r], h_bits[r]);
-        if (k < 0) return RMSMP_ERR_SCHEME;
-        ++cnt[k];
-    }
     std::memset(L, 0, sizeof(*L));
     L->magic = kLayerMagic;
     L->M = M; L->Cin = Cin; L->kh = kh; L->kw = kw;
@@ -262,15 +255,6 @@ rmsmp_status rmsmp_layer_init(rmsmp_layer* L, int M, int Cin, int kh, int kw,
     if (kh * kw > 1 && L->Kp > 196608) return RMSMP_ERR_SHAPE;   // one shared-memory segment in the pack kernel
     L->nP = cnt[0]; L->nF4 = cnt[1]; L->n8 = cnt[2];
     L->nblocks = (M + kBlockRows - 1) / kBlockRows;
-    // bytes one k-block of one block's packed rows takes when fetched group by group in 16-row boxes
-    int raw_max = 0;
-    for (int b0 = 0; b0 < M; b0 += kBlockRows) {
-        int c[3] = {0, 0, 0};
-        for (int r = b0; r < M && r < b0 + kBlockRows; ++r) ++c[row_kind(h_scheme[r], h_bits[r])];
-        const int bytes = ((c[0] + 15) / 16 * 16 + (c[1] + 15) / 16 * 16) * 64 + (c[2] + 15) / 16 * 16 * 128;
-        raw_max = std::max(raw_max, bytes);
-    }
-    L->raw_stage_bytes = raw_max;
     uint64_t off = 256;
     L->off_perm = off;   off = align_up(off + 4ull * M, 256);
     L->off_slot = off;   off = align_up(off + 4ull * M, 256);
@@ -281,6 +265,90 @@ rmsmp_status rmsmp_layer_init(rmsmp_layer* L, int M, int Cin, int kh, int kw,
     L->off_q4 = off;     off = align_up(off + (uint64_t)(cnt[0] + cnt[1]) * (L->Kp / 2), 256);
     L->off_q8 = off;     off = align_up(off + (uint64_t)cnt[2] * L->Kp, 256);
     L->packed_bytes = off;
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_layer_init(rmsmp_layer* L, int M, int Cin, int kh, int kw,
+                              const uint8_t* h_scheme, const uint8_t* h_bits)
+{
+    if (!L || !h_scheme || !h_bits) return RMSMP_ERR_NULL;
+    if (M < 1 || M > (1 << 20)) return RMSMP_ERR_SHAPE;
+    int cnt[3] = {0, 0, 0};
+    for (int r = 0; r < M; ++r) {
+        const int k = row_kind(h_scheme[r], h_bits[r]);
+        if (k < 0) return RMSMP_ERR_SCHEME;
+        ++cnt[k];
+    }
+    rmsmp_status s = layer_layout(L, M, Cin, kh, kw, cnt);
+    if (s != RMSMP_OK) return s;
+    // bytes one k-block of one block's packed rows takes when fetched group by group in 16-row boxes
+    int raw_max = 0;
+    for (int b0 = 0; b0 < M; b0 += kBlockRows) {
+        int c[3] = {0, 0, 0};
+        for (int r = b0; r < M && r < b0 + kBlockRows; ++r) ++c[row_kind(h_scheme[r], h_bits[r])];
+        const int bytes = ((c[0] + 15) / 16 * 16 + (c[1] + 15) / 16 * 16) * 64 + (c[2] + 15) / 16 * 16 * 128;
+        raw_max = std::max(raw_max, bytes);
+    }
+    L->raw_stage_bytes = raw_max;
+    return RMSMP_OK;
+}
+
+static void ratio_counts(int M, int A, int C, int cnt[3])
+{
+    int n8 = (int)std::floor((double)M * C / 100.0 + 0.5);
+    n8 = std::min(n8, M);
+    int nP = (int)std::floor((double)M * A / 100.0 + 0.5);
+    nP = std::min(nP, M - n8);
+    cnt[0] = nP; cnt[1] = M - nP - n8; cnt[2] = n8;
+}
+
+rmsmp_status rmsmp_layer_init_ratio(rmsmp_layer* L, int M, int Cin, int kh, int kw, int A, int B, int C)
+{
+    if (!L) return RMSMP_ERR_NULL;
+    if (M < 1 || M > 65536 || A < 0 || B < 0 || C < 0 || A + B + C != 100) return RMSMP_ERR_SHAPE;
+    int cnt[3];
+    ratio_counts(M, A, C, cnt);
+    rmsmp_status s = layer_layout(L, M, Cin, kh, kw, cnt);
+    if (s != RMSMP_OK) return s;
+    // which rows share a 128-row block is not known before the weights are ranked: the most a block can need
+    auto up16 = [](int n) { return (n + 15) / 16 * 16; };
+    L->raw_stage_bytes = (up16(std::min(kBlockRows, cnt[0])) + up16(std::min(kBlockRows, cnt[1]))) * 64 +
+                         up16(std::min(kBlockRows, cnt[2])) * 128;
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_assign_scratch_bytes(int M, size_t* bytes)
+{
+    if (!bytes) return RMSMP_ERR_NULL;
+    if (M < 1 || M > 65536) return RMSMP_ERR_SHAPE;
+    *bytes = assign_scratch_bytes(M);
+    return RMSMP_OK;
+}
+
+rmsmp_status rmsmp_assign_quantize_pack(const float* d_W, rmsmp_w_layout w_layout, const rmsmp_layer* L, int A, int B,
+                                        int C, const float* d_alpha, rmsmp_pot_mode pot_mode, void* d_packed,
+                                        size_t packed_bytes, void* d_scratch, size_t scratch_bytes, uint8_t* d_scheme,
+                                        uint8_t* d_bits, void* stream)
+{
+    if (!d_W || !L || !d_packed || !d_scratch) return RMSMP_ERR_NULL;
+    if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+    if (L->M > 65536 || A < 0 || B < 0 || C < 0 || A + B + C != 100) return RMSMP_ERR_SHAPE;
+    if (w_layout != RMSMP_W_LINEAR && w_layout != RMSMP_W_CONV_OIHW) return RMSMP_ERR_SHAPE;
+    if (w_layout == RMSMP_W_LINEAR && (L->kh != 1 || L->kw != 1)) return RMSMP_ERR_SHAPE;
+    if (pot_mode != RMSMP_POT_NEAREST && pot_mode != RMSMP_POT_LOG2) return RMSMP_ERR_SCHEME;
+    int cnt[3];
+    ratio_counts(L->M, A, C, cnt);
+    if (cnt[0] != L->nP || cnt[1] != L->nF4 || cnt[2] != L->n8) return RMSMP_ERR_SCHEME;   // descriptor of another ratio
+    if (packed_bytes < L->packed_bytes || scratch_bytes < assign_scratch_bytes(L->M)) return RMSMP_ERR_BUFFER_TOO_SMALL;
+    if (!aligned16(d_W) || (reinterpret_cast<uintptr_t>(d_packed) & 255) != 0 || !aligned16(d_scratch)) return RMSMP_ERR_ALIGN;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (launch_assign_meta(d_W, *L, d_alpha, pot_mode, static_cast<uint8_t*>(d_packed), d_scratch, d_scheme, d_bits, st) != cudaSuccess ||
+        launch_pack(d_W, w_layout == RMSMP_W_CONV_OIHW, *L, pot_mode, static_cast<uint8_t*>(d_packed), st) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
     return RMSMP_OK;
 }
 

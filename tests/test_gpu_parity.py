@@ -530,3 +530,45 @@ def test_a_bounded_wait_that_runs_out_reports_timeout_and_leaves_the_context_usa
     _, _, acc_ref, y_ref = O.layer_linear(Wt, scheme, bits, alpha, act, np.float32(0.25))
     assert np.array_equal(acc, acc_ref)
     assert np.array_equal(y.view(np.uint32), y_ref.view(np.uint32))
+
+
+# ------------------------------------------------------------------ row assignment on the device
+
+@pytest.mark.parametrize("ratio", [(60, 35, 5), (65, 30, 5), (0, 100, 0), (50, 40, 10)], ids=lambda r: "%d-%d-%d" % r)
+@pytest.mark.parametrize("shape", [(256, 512), (130, 96), (1000, 2304), (64, 64, 3, 3), (160, 48, 3, 3)], ids=str)
+def test_assignment_on_the_device_matches_oracle(shape, ratio):
+    """Ratio in, packed layer out: the assignment (variance rank), the grouping, the per-row steps and every
+    code must equal the oracle's assign_rows -> quantize_rows -> group_rows; then the layer runs."""
+    import torch
+    g = synth.rng(85, sum(shape) + ratio[0])
+    conv = len(shape) == 4
+    Wt = synth.weights_kaiming(g, *shape) if conv else synth.weights_normal(g, shape)
+    if not conv:
+        Wt[7] = Wt[3]                                   # two rows of equal variance: the row index decides
+    M = shape[0]
+    Cin, kh, kw = (shape[1], shape[2], shape[3]) if conv else (shape[1], 1, 1)
+    layer = R.rmsmp_layer_init_ratio(M, Cin, kh, kw, ratio)
+    d_W = torch.from_numpy(Wt).cuda()
+    d_packed = torch.empty(layer.packed_bytes, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(R.rmsmp_assign_scratch_bytes(M), dtype=torch.uint8, device="cuda")
+    d_scheme = torch.empty(M, dtype=torch.uint8, device="cuda")
+    d_bits = torch.empty(M, dtype=torch.uint8, device="cuda")
+    R.rmsmp_assign_quantize_pack(d_W, R.W_CONV_OIHW if conv else R.W_LINEAR, layer, ratio, None, R.POT_NEAREST, d_packed,
+                                 scratch, d_scheme, d_bits)
+    torch.cuda.synchronize()
+    scheme, bits = O.assign_rows(Wt, ratio)
+    assert np.array_equal(d_scheme.cpu().numpy(), scheme) and np.array_equal(d_bits.cpu().numpy(), bits)
+    alpha = synth.alpha_rows(Wt)
+    v_ref, ws_ref = O.quantize_rows(Wt.reshape(M, -1), scheme, bits, alpha)
+    vals, perm, ws = Hn.unpack(layer, d_packed)
+    assert np.array_equal(perm, O.group_rows(scheme, bits))
+    assert np.array_equal(ws.view(np.uint32), ws_ref.view(np.uint32))
+    assert np.array_equal(vals, v_ref)
+    # the same descriptor as the host route gives, and a layer run on top of it
+    ref_layer = R.rmsmp_layer_init(M, Cin, kh, kw, scheme, bits)
+    assert (layer.nP, layer.nF4, layer.n8, layer.packed_bytes) == (ref_layer.nP, ref_layer.nF4, ref_layer.n8, ref_layer.packed_bytes)
+    if not conv:
+        act = synth.act_codes_uniform(g, (77, shape[1]))
+        for variant in (R.VARIANT_AUTO, R.VARIANT_TENSOR if shape[1] % 16 == 0 else R.VARIANT_SIMT, Hn.WORKSPACE if shape[1] % 16 == 0 else R.VARIANT_SIMT):
+            y, acc = Hn.gemm(layer, d_packed, act, 0.05, variant)
+            assert np.array_equal(acc, O.matmul(v_ref, act))
