@@ -232,6 +232,21 @@ rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* layer, const void* d
                                          rmsmp_variant variant, void* stream);
 
 /*
+ * Depthwise convolution (the 3x3 layers of MobileNet-v2, one of the paper's models, Section 4.1): every
+ * channel is convolved with its own filter, and every filter is a weight row with its own scheme and
+ * precision (Figure 2).  The layer is described and packed like any other with M = channels and Cin = 1
+ * (weights [C][1][kh][kw]); activation codes d_act are [B][H][W][C], results
+ *   acc[b][ho][wo][c] = sum_{i,j} value[c][i][j] * act[b][ho*stride+i-pad][wo*stride+j-pad][c]   (zero outside)
+ *   y = (float)acc * (wstep[c] * act_step)
+ * in [B][Ho][Wo][C]; d_acc optional.  CUDA cores (there is no contraction over channels).
+ * Errors: NULL, BAD_LAYER, SHAPE (layer not Cin = 1, bad geometry), SCALE, ALIGN, ARCH, CUDA; VARIANT when C is
+ * not a multiple of 4 or the filters do not fit shared memory (kh * kw * C > 51,200).
+ */
+rmsmp_status rmsmp_conv_depthwise(const rmsmp_layer* layer, const void* d_packed, const int8_t* d_act, int B,
+                                  int H, int W, int stride, int pad, float act_step, float* d_out,
+                                  int32_t* d_acc, void* stream);
+
+/*
  * Many small-batch linear layers in one launch (Algorithm 1's forward line, layer after layer;
  * Section 3.1: the layers execute one after another on the same hardware).  With a
  * handful of tokens a layer is bound by reading its packed weights once, which takes a fraction

@@ -322,6 +322,36 @@ void rmsmp_o_conv(const int8_t *v, const int8_t *a, int M, int Cin, int kh, int 
                 }
 }
 
+/*
+ * Depthwise convolution (MobileNet-v2, one of the paper's models, Section 4.1; every filter is a
+ * weight row of its own, Figure 2): channel c of the output sees channel c of the input only.
+ * v[C][kh][kw], a[B][H][W][C], zero outside the image, acc[B][Ho][Wo][C].
+ */
+void rmsmp_o_conv_depthwise(const int8_t *v, const int8_t *a, int C, int kh, int kw,
+                            int B, int H, int W, int stride, int pad, int32_t *acc)
+{
+    int Ho = (H + 2 * pad - kh) / stride + 1;
+    int Wo = (W + 2 * pad - kw) / stride + 1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int ho = 0; ho < Ho; ++ho)
+            for (int wo = 0; wo < Wo; ++wo)
+                for (int c = 0; c < C; ++c) {
+                    int32_t s = 0;
+                    for (int i = 0; i < kh; ++i) {
+                        int y = ho * stride + i - pad;
+                        if (y < 0 || y >= H) continue;
+                        for (int j = 0; j < kw; ++j) {
+                            int x = wo * stride + j - pad;
+                            if (x < 0 || x >= W) continue;
+                            s += (int32_t)v[((size_t)c * kh + i) * kw + j] *
+                                 (int32_t)a[(((size_t)b * H + y) * W + x) * C + c];
+                        }
+                    }
+                    acc[(((size_t)b * Ho + ho) * Wo + wo) * C + c] = s;
+                }
+}
+
 /* One output of the convolution at a time: (pixel index n = (b*Ho+ho)*Wo+wo, row r). */
 void rmsmp_o_conv_points(const int8_t *v, const int8_t *a, int M, int Cin, int kh, int kw,
                          int B, int H, int W, int stride, int pad, const int64_t *n_idx,

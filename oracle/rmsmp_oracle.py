@@ -170,6 +170,18 @@ def conv(values, act, stride: int, pad: int) -> np.ndarray:
     return acc
 
 
+def conv_depthwise(values, act, stride: int, pad: int) -> np.ndarray:
+    """values[C][kh][kw] int8, act[B][H][W][C] int8 -> acc[B][Ho][Wo][C] int32 (each channel with its own filter)."""
+    values, act = _c(values, np.int8), _c(act, np.int8)
+    Cc, kh, kw = values.shape
+    B, H, W, Ca = act.shape
+    assert Ca == Cc
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad)
+    acc = np.empty((B, Ho, Wo, Cc), np.int32)
+    lib().rmsmp_o_conv_depthwise(_p(values), _p(act), Cc, kh, kw, B, H, W, stride, pad, _p(acc))
+    return acc
+
+
 def conv_points(values, act, stride: int, pad: int, n_idx, r_idx) -> np.ndarray:
     values, act = _c(values, np.int8), _c(act, np.int8)
     M, Cin, kh, kw = values.shape

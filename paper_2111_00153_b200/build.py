@@ -8,7 +8,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "librmsmp.so")
-SOURCES = ("host_api.cu", "pack.cu", "simt.cu", "tensor.cu", "tensor2.cu", "peak.cu", "builtin_scratch.cu", "stream.cu", "assign.cu")
+SOURCES = ("host_api.cu", "pack.cu", "simt.cu", "tensor.cu", "tensor2.cu", "peak.cu", "builtin_scratch.cu", "stream.cu", "assign.cu", "depthwise.cu")
 HEADERS = tuple(sorted(f for f in os.listdir(CSRC) if f.endswith((".cuh", ".h")))) + \
           (os.path.join("..", "..", "include", "rmsmp.h"),)
 

@@ -87,6 +87,9 @@ rmsmp_status dispatch_problem(Problem& p, rmsmp_variant variant, cudaStream_t st
 // kernels (each returns the CUDA launch error, cudaSuccess if fine)
 cudaError_t launch_pack(const float* dW, int conv_oihw, const rmsmp_layer& L, int pot_mode,
                         uint8_t* blob, cudaStream_t st);
+// depthwise convolution on the CUDA cores (depthwise.cu)
+bool depthwise_supported(const Problem& p);
+cudaError_t launch_depthwise(const Problem& p, cudaStream_t st);
 // row assignment on the device + the packed buffer's metadata (assign.cu); scratch of assign_scratch_bytes(M)
 size_t assign_scratch_bytes(int M);
 cudaError_t launch_assign_meta(const float* dW, const rmsmp_layer& L, const float* d_alpha, int pot_mode, uint8_t* blob,

@@ -715,6 +715,36 @@ static rmsmp_status conv_impl(const rmsmp_layer* L, const void* d_packed, const 
     return dispatch(p, variant, static_cast<cudaStream_t>(stream));
 }
 
+rmsmp_status rmsmp_conv_depthwise(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act, int B, int H, int W,
+                                  int stride, int pad, float act_step, float* d_out, int32_t* d_acc, void* stream)
+{
+    if (!L || !d_packed || !d_act || !d_out) return RMSMP_ERR_NULL;
+    if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
+    if (L->Cin != 1) return RMSMP_ERR_SHAPE;              // a depthwise layer is described as M = channels, Cin = 1
+    if (B < 1 || H < 1 || W < 1 || stride < 1 || stride > 8 || pad < 0 || pad > 16) return RMSMP_ERR_SHAPE;
+    if (H + 2 * pad < L->kh || W + 2 * pad < L->kw) return RMSMP_ERR_SHAPE;
+    if (!std::isfinite(act_step)) return RMSMP_ERR_SCALE;
+    const int Ho = (H + 2 * pad - L->kh) / stride + 1, Wo = (W + 2 * pad - L->kw) / stride + 1;
+    const int64_t N = (int64_t)B * Ho * Wo;
+    if (N > (int64_t)1 << 31 || (int64_t)B * H * W > (int64_t)1 << 31) return RMSMP_ERR_SHAPE;
+    if (!aligned16(d_act) || !aligned16(d_out) || (d_acc && !aligned16(d_acc)) || (reinterpret_cast<uintptr_t>(d_packed) & 255))
+        return RMSMP_ERR_ALIGN;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    Problem p;
+    fill_problem(p, L, d_packed);
+    p.act = d_act;
+    p.B = B; p.H = H; p.W = W; p.Ho = Ho; p.Wo = Wo; p.stride = stride; p.pad = pad;
+    p.pix_pitch = L->M; p.N = N;                          // channels last: a pixel holds one code per channel
+    p.act_step = act_step; p.out = d_out; p.acc = d_acc; p.out_mn = 0; p.ld_out = L->M;
+    if (!depthwise_supported(p)) return RMSMP_ERR_VARIANT;
+    if (launch_depthwise(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return RMSMP_OK;
+}
+
 rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* L, const void* d_packed,
                                          const int8_t* d_act, int B, int H, int W, int stride,
                                          int pad, float act_step, float* d_out,

@@ -572,3 +572,52 @@ def test_assignment_on_the_device_matches_oracle(shape, ratio):
         for variant in (R.VARIANT_AUTO, R.VARIANT_TENSOR if shape[1] % 16 == 0 else R.VARIANT_SIMT, Hn.WORKSPACE if shape[1] % 16 == 0 else R.VARIANT_SIMT):
             y, acc = Hn.gemm(layer, d_packed, act, 0.05, variant)
             assert np.array_equal(acc, O.matmul(v_ref, act))
+
+
+# ------------------------------------------------------------------ depthwise convolution
+
+@pytest.mark.parametrize("C,k,stride,pad,B,H,W,kind", [
+    (32, 3, 1, 1, 2, 14, 14, R.ACT_U4),
+    (96, 3, 2, 1, 3, 15, 13, R.ACT_U4),        # MobileNet-v2 style stride-2 block, odd sizes
+    (144, 3, 1, 1, 1, 28, 28, R.ACT_S4),
+    (960, 3, 1, 1, 2, 7, 7, R.ACT_U4),         # the widest depthwise layer of MobileNet-v2
+    (8, 5, 1, 2, 2, 6, 9, R.ACT_S4),
+])
+def test_depthwise_conv_matches_oracle(C, k, stride, pad, B, H, W, kind):
+    import torch
+    g = synth.rng(86, C + k + H)
+    Wt = synth.weights_kaiming(g, C, 1, k, k)
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    alpha = synth.alpha_rows(Wt)
+    x = synth.act_halfnormal(g, (B, H, W, C)) if kind == R.ACT_U4 else synth.act_normal(g, (B, H, W, C))
+    codes, act_step = O.quantize_act(x, synth.ALPHA_ACT, kind)
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, alpha)
+    v_ref, wstep = O.quantize_rows(Wt.reshape(C, -1), scheme, bits, alpha)
+    acc_ref = O.conv_depthwise(v_ref.reshape(C, k, k), codes, stride, pad)
+    y_ref = O.epilogue(acc_ref, wstep, act_step)
+    Ho, Wo = O.conv_out_hw(H, W, k, k, stride, pad)
+    y = torch.full((B, Ho, Wo, C), float("nan"), dtype=torch.float32, device="cuda")
+    acc = torch.full((B, Ho, Wo, C), -5, dtype=torch.int32, device="cuda")
+    R.rmsmp_conv_depthwise(layer, d_packed, torch.from_numpy(codes).cuda(), B, H, W, stride, pad, float(act_step), y, acc)
+    torch.cuda.synchronize()
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
+
+
+def test_depthwise_conv_rejects_what_it_cannot_run():
+    import torch
+    g = synth.rng(86, 1)
+    Wt = synth.weights_kaiming(g, 6, 1, 3, 3)            # 6 channels: not a multiple of 4
+    scheme, bits = O.assign_rows(Wt, (60, 35, 5))
+    layer, d_packed = Hn.pack_layer(Wt, scheme, bits, synth.alpha_rows(Wt))
+    a = torch.zeros((1, 4, 4, 8), dtype=torch.int8, device="cuda")
+    y = torch.zeros((1, 4, 4, 8), dtype=torch.float32, device="cuda")
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_conv_depthwise(layer, d_packed, a, 1, 4, 4, 1, 1, 0.1, y)
+    assert e.value.status == R.ERR_VARIANT
+    Wd = synth.weights_kaiming(g, 8, 2, 3, 3)            # an ordinary layer is not a depthwise one
+    scheme, bits = O.assign_rows(Wd, (60, 35, 5))
+    layer, d_packed = Hn.pack_layer(Wd, scheme, bits, synth.alpha_rows(Wd))
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_conv_depthwise(layer, d_packed, a, 1, 4, 4, 1, 1, 0.1, y)
+    assert e.value.status == R.ERR_SHAPE

@@ -409,3 +409,26 @@ def test_op_count_convention_matches_table6():
     macs += synth.RESNET18_CONV1.macs(1) + synth.RESNET18_FC_MACS
     assert abs(2 * macs / 1e9 - float(np.median(prods))) < 0.03
     assert sum(L.count for L in synth.resnet18_convs()) == 19
+
+
+def test_depthwise_conv_is_the_dense_conv_with_block_diagonal_filters():
+    """Pin of the depthwise oracle: the same sums as the ordinary convolution when filter c is zero on
+    every input channel but c (the definition of a depthwise layer), at three geometries; and one
+    output re-added by hand."""
+    g = np.random.default_rng(11)
+    for (Cc, k, stride, pad, B, H, W) in ((8, 3, 1, 1, 2, 6, 7), (12, 3, 2, 1, 1, 9, 8), (4, 5, 1, 2, 2, 5, 5)):
+        v = g.integers(-127, 128, size=(Cc, k, k)).astype(np.int8)
+        a = g.integers(-7, 16, size=(B, H, W, Cc)).astype(np.int8)
+        dense = np.zeros((Cc, Cc, k, k), np.int8)
+        for c in range(Cc):
+            dense[c, c] = v[c]
+        got = O.conv_depthwise(v, a, stride, pad)
+        assert np.array_equal(got, O.conv(dense, a, stride, pad))
+        b, ho, wo, c = B - 1, 1, 2, Cc - 1
+        s = 0
+        for i in range(k):
+            for j in range(k):
+                y, x = ho * stride + i - pad, wo * stride + j - pad
+                if 0 <= y < H and 0 <= x < W:
+                    s += int(v[c, i, j]) * int(a[b, y, x, c])
+        assert got[b, ho, wo, c] == s
