@@ -414,6 +414,7 @@ def run_ours(args):
                              "layers": len(tb)} if tb and i8_peak > 0 else None),
         "roofline_weights": (weights_leg(R, torch, peaks) if (world == 1 and not args.no_weights_leg) else None),
         "per_config": (configs_leg(R, torch, peaks, i8_peak) if (world == 1 and not args.no_weights_leg and i8_peak > 0) else None),
+        "second_workloads": (second_workloads_leg(R, torch, peaks, i8_peak) if (world == 1 and not args.no_weights_leg and i8_peak > 0) else None),
         "roofline_per_layer": binding_roof_summary(H, conv_ms_layer, alg, batch, peaks["hbm_gbs"], i8_peak, peaks),
         "per_layer": [{"name": h["L"].name, "M": h["L"].M, "K": h["L"].K, "N": d["N"], "ms": float(ms),
                        "tops": layer_ops(h["L"], batch) / (ms * 1e-3) / 1e12, "gbs": float(a / (ms * 1e-3) / 1e9)}
@@ -494,7 +495,72 @@ def configs_leg(R, torch, peaks, i8_peak):
     return rows
 
 
-def weights_leg(R, torch, peaks, tokens=(1, 8, 128), reps=5, launches=20):
+def second_workloads_leg(R, torch, peaks, i8_peak):
+    """Layer shapes of the paper's other models (Section 4.1: MobileNet-v2, ResNet-50) and ResNet-18's first
+    layer: depthwise 3x3 (CUDA cores), pointwise / bottleneck 1x1 and the 7x7 stride-2 first convolution
+    with its three input channels stored as 16 (tensor cores).  Batch 64; 20 replays between two events."""
+    rows = []
+
+    def timed(fn):
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(20):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) / 20)
+        return float(np.median(ts))
+
+    def pack(W):
+        scheme, bits = R.rmsmp_assign_rows(W, RATIO)
+        lay = R.rmsmp_layer_init(W.shape[0], W.shape[1], W.shape[2], W.shape[3], scheme, bits)
+        pk = torch.empty(lay.packed_bytes, dtype=torch.uint8, device="cuda")
+        R.rmsmp_quantize_pack(torch.from_numpy(W).cuda(), R.W_CONV_OIHW, lay, scheme, bits, synth.alpha_rows(W), R.POT_NEAREST, pk)
+        return lay, pk
+
+    def record(name, lay, ms, ops, alg):
+        t_h, t_t = alg / (peaks["hbm_gbs"] * 1e9) * 1e3, ops / (i8_peak * 1e12) * 1e3
+        rows.append({"shape": name, "us": ms * 1e3, "tops": ops / (ms * 1e-3) / 1e12, "gbs": alg / (ms * 1e-3) / 1e9,
+                     "bound": "tensor" if t_t > t_h else "hbm", "frac": max(t_h, t_t) / ms})
+
+    B = 64
+    for (C, H, stride) in ((144, 56, 1), (192, 28, 2), (960, 7, 1)):
+        W = synth.weights_kaiming(synth.rng(7, C + H), C, 1, 3, 3)
+        lay, pk = pack(W)
+        Ho = (H + 2 - 3) // stride + 1
+        act = torch.randint(0, 16, (B, H, H, C), dtype=torch.int8, device="cuda")
+        y = torch.empty((B, Ho, Ho, C), dtype=torch.float32, device="cuda")
+        ms = timed(lambda: R.rmsmp_conv_depthwise(lay, pk, act, B, H, H, stride, 1, 0.1, y))
+        N = B * Ho * Ho
+        record("mobilenet-v2 depthwise 3x3 C=%d %dx%d s%d B=%d" % (C, H, H, stride, B), lay, ms, 2 * 9 * C * N,
+               lay.packed_bytes + B * H * H * C + 4 * N * C)
+    for (name, M, Cin, k, stride, pad, H) in (("mobilenet-v2 pointwise 1x1 32->192 28x28", 192, 32, 1, 1, 0, 28),
+                                              ("resnet-50 bottleneck 1x1 256->64 56x56", 64, 256, 1, 1, 0, 56),
+                                              ("resnet-50 bottleneck 1x1 64->256 56x56", 256, 64, 1, 1, 0, 56),
+                                              ("resnet-18 conv1 7x7 s2 (3 channels stored as 16) 224x224", 64, 16, 7, 2, 3, 224)):
+        W = synth.weights_kaiming(synth.rng(7, M + Cin + k), M, Cin, k, k)
+        if k == 7:
+            W[:, 3:] = 0.0
+        lay, pk = pack(W)
+        ws = torch.empty(R.rmsmp_workspace_bytes(lay), dtype=torch.int8, device="cuda")
+        R.rmsmp_expand_weights(lay, pk, ws)
+        Ho = (H + 2 * pad - k) // stride + 1
+        N = B * Ho * Ho
+        act = torch.randint(0, 16, (B, H, H, Cin), dtype=torch.int8, device="cuda")
+        y = torch.empty((N, M), dtype=torch.float32, device="cuda")
+        ms = timed(lambda: R.rmsmp_conv_implicit_workspace(lay, pk, ws, act, B, H, H, stride, pad, 0.1, y, R.OUT_NM, None))
+        real_cin = 3 if k == 7 else Cin
+        record(name + " B=%d" % B, lay, ms, 2 * M * real_cin * k * k * N,
+               (lay.nP + lay.nF4) * real_cin * k * k // 2 + lay.n8 * real_cin * k * k + 8 * M + B * H * H * real_cin + 4 * N * M)
+    return rows
+
+
+def weights_leg(R, torch, peaks, tokens=(1, 8, 128), reps=5, launches=20, warm=50):
     """The weight-bound regime (config 5): the whole BERT-large stack (144 linears, ~160 MB of packed codes,
     more than L2) through ONE grouped tensor-core launch per pass, at a few token counts.  The plan is
     prepared once; a pass is one launch; `launches` passes run back to back between two events."""
@@ -516,7 +582,7 @@ def weights_leg(R, torch, peaks, tokens=(1, 8, 128), reps=5, launches=20):
         arr = R.make_gemm_items(items)
         table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
         plan = R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table)
-        for _ in range(50):
+        for _ in range(warm):
             R.rmsmp_gemm_grouped_launch(plan)
         torch.cuda.synchronize()
         best = []
@@ -564,7 +630,7 @@ def binding_roof_summary(H, ms_layer, alg_bytes, batch, hbm_gbs, i8_peak, peaks)
 
 
 TRAFFIC_NOTE = os.path.join(ROOT, "profiles", "resnet18_stack_dram_traffic.txt")
-KERNEL_SOURCES = ("tensor.cu", "tensor2.cu", "common.cuh", "decode.cuh", "actq.cuh")
+KERNEL_SOURCES = ("tensor.cu", "tensor2.cu", "common.cuh", "decode.cuh", "actq.cuh", "ptx.cuh", "tmap.cuh")
 
 
 def kernel_sources_digest():
@@ -588,6 +654,40 @@ def measured_traffic():
         return float(kv["dram_bytes_per_step"])
     except Exception:
         return None
+
+
+def write_traffic_note(csv_path):
+    """Turns the profiler's launch list (ncu --csv with gpu__time_duration.sum, dram__bytes_read.sum and
+    dram__bytes_write.sum per launch, taken on `bench.py --steps 2 --warmup 3 --no-e2e --no-cpu-baseline
+    --no-weights-leg`) into the note measured_traffic() reads: the DRAM bytes of the 19 convolution launches
+    of one whole step, tied to the digest of the kernels' sources."""
+    import collections
+    import csv
+    rows = [r for r in csv.reader(open(csv_path)) if len(r) > 10]
+    hdr = rows[0]
+    ik, im, iv, iid = hdr.index("Kernel Name"), hdr.index("Metric Name"), hdr.index("Metric Value"), hdr.index("ID")
+    per = collections.OrderedDict()
+    for r in rows[1:]:
+        per.setdefault(r[iid], {"name": r[ik]})[r[im]] = float(r[iv].replace(",", ""))
+    conv = [v for v in per.values() if "tensor_kernel" in v["name"] or "pair_kernel" in v["name"]]
+    first_form = conv[0]["name"] if conv else ""
+    n_layers = len(layer_list())
+    # a step starts with the first layer's kernel form after a different one (the l1 layers open the stack)
+    l1 = next(v["name"] for v in conv if "pair_kernel" not in v["name"] and ", 3, " in v["name"])
+    start = next(i for i in range(1, len(conv) - n_layers) if conv[i]["name"] == l1 and conv[i - 1]["name"] != l1)
+    step = conv[start:start + n_layers]
+    total = sum(v["dram__bytes_read.sum"] + v["dram__bytes_write.sum"] for v in step)
+    us = sum(v["gpu__time_duration.sum"] for v in step) / 1e3
+    with open(TRAFFIC_NOTE, "w") as f:
+        f.write("# DRAM traffic of the %d convolution launches of one step (ResNet-18 stack, batch 256), from the profiler's\n" % n_layers)
+        f.write("# launch list: ncu --metrics gpu__time_duration.sum,dram__bytes_read.sum,dram__bytes_write.sum --clock-control none\n")
+        f.write("#   -s 200 -c 200 --csv --log-file gpurun_out/launches.csv python bench.py --steps 2 --warmup 3 --no-e2e --no-cpu-baseline --no-weights-leg\n")
+        f.write("# then: python bench.py --write-traffic-note gpurun_out/launches.csv\n")
+        f.write("kernel_sources_sha256: %s\n" % kernel_sources_digest())
+        f.write("dram_bytes_per_step: %.0f\n" % total)
+        f.write("conv_launches: %d\n" % len(step))
+        f.write("conv_time_under_profiler_us: %.1f\n" % us)
+    print(open(TRAFFIC_NOTE).read())
 
 
 def load_peaks():
@@ -852,6 +952,10 @@ def main():
     ap.add_argument("--suite-filter", default=None,
                     help="with --suite: only the rows whose configuration tag contains this text "
                          "(config1 .. config5, or 'grouped' for the one-launch BERT-large stack)")
+    ap.add_argument("--weights-leg-only", default=None, metavar="TOKENS",
+                    help="run only the weight-bound leg at this token count and print it (short: for profiler captures)")
+    ap.add_argument("--write-traffic-note", default=None, metavar="CSV",
+                    help="no GPU work: turn a profiler launch list into the DRAM-traffic note roofline.traffic is read from")
     ap.add_argument("--check-ranks", action="store_true",
                     help="no GPU work: the ranks check their seeding and the max-over-ranks exchange over gloo")
     ap.add_argument("--layers", default=None,
@@ -862,7 +966,15 @@ def main():
         LAYER_FILTER = set(args.layers.split(","))
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.suite:
         sys.exit(launch_ranks(sys.argv[1:], args.gpus))
-    if args.check_ranks:
+    if args.write_traffic_note:
+        write_traffic_note(args.write_traffic_note)
+    elif args.weights_leg_only:
+        import torch
+        from paper_2111_00153_b200 import binding as R
+        torch.cuda.set_device(0)
+        peaks, _ = load_peaks()
+        print(json.dumps(weights_leg(R, torch, peaks, tokens=(int(args.weights_leg_only),), reps=2, launches=3, warm=3)))
+    elif args.check_ranks:
         run_check_ranks(args)
     elif args.suite:
         run_suite(args)
