@@ -582,6 +582,8 @@ def test_assignment_on_the_device_matches_oracle(shape, ratio):
     (144, 3, 1, 1, 1, 28, 28, R.ACT_S4),
     (960, 3, 1, 1, 2, 7, 7, R.ACT_U4),         # the widest depthwise layer of MobileNet-v2
     (8, 5, 1, 2, 2, 6, 9, R.ACT_S4),
+    (1280, 3, 1, 1, 1, 5, 6, R.ACT_S4),        # more channel quads than threads of a block
+    (16, 3, 3, 0, 2, 11, 10, R.ACT_U4),        # a stride the run kernel does not take
 ])
 def test_depthwise_conv_matches_oracle(C, k, stride, pad, B, H, W, kind):
     import torch
