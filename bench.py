@@ -574,7 +574,7 @@ def weights_leg(R, torch, peaks, tokens=(1, 8, 128), reps=5, launches=20, warm=5
             act = torch.from_numpy(synth.act_codes_uniform(g, (N, K))).cuda()
             y = torch.empty((N, M), dtype=torch.float32, device="cuda")
             keep.append((act, y))
-            items.append((lay, pk, act, N, K, 0.1, y, M, None))
+            items.append((lay, pk, act, N, K, 0.1, y, M, None, 1))      # codes 0..15: act_nonneg
             w = (lay.nP + lay.nF4) * K // 2 + lay.n8 * K + 8 * M
             wbytes += w
             alg += w + N * K + 4 * N * M

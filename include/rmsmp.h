@@ -269,6 +269,9 @@ typedef struct rmsmp_gemm_item {
     float* d_out;
     int64_t ld_out;
     int32_t* d_acc;            /* optional */
+    int32_t act_nonneg;        /* tensor-core grouped launch only: nonzero = the caller guarantees that every
+                                  activation code is within 0..15 (the unsigned 4-bit activations of Eq. 1);
+                                  0 = codes may be negative (within -16..16) */
 } rmsmp_gemm_item;
 rmsmp_status rmsmp_grouped_table_bytes(int count, size_t* bytes);
 rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
@@ -278,17 +281,30 @@ rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp
  * The same grouped launch on the tensor cores, split into a set-up call and a launch call
  * (Section 3.1: rows of every scheme streamed to their cores and finishing together; here all
  * layers' packed rows stream through the SMs in one kernel).  One persistent CTA per SM takes
- * blocks of 128 rows of any layer, fetches their packed codes with TMA, expands them to int8 in
- * registers, hands them to the tensor cores through tensor memory and multiplies them with up to
- * 128 tokens on tcgen05 (int32 accumulators in tensor memory).  Results are bit for bit those of
- * rmsmp_gemm.
- *   rmsmp_grouped_plan_bytes    scratch size for the table of these layers on the current device.
+ * blocks of 128 rows of one kind of any layer, fetches their packed codes with TMA, expands them
+ * in registers, hands them to the tensor cores through tensor memory and multiplies them with up
+ * to 128 tokens on tcgen05.  Fixed-4 and Fixed-8 rows become int8 operands with int32 sums.  A
+ * PoT-4 code (Eq. 4: sign and exponent) shifted left by two is the 6-bit float of a quarter of its
+ * value, so PoT rows go to the tensor core's float path as they are (E3M2 weights x E4M3
+ * activations, fp32 sums); every product and partial sum is a multiple of 1/4 below 2^22, which
+ * fp32 holds exactly.  The activation bytes of a layer whose item says act_nonneg are read as
+ * they are: a byte 0..15 taken as an E4M3 number is that code times 2^-9.  Otherwise the launch
+ * first writes an E4M3 copy of the layer's codes into scratch behind the table.  Results are bit
+ * for bit those of rmsmp_gemm for activation codes within -16..16 (the 4-bit codes of Eq. 1/Eq. 3,
+ * signed or unsigned; 0..15 with act_nonneg); other int8 values are not supported by this entry
+ * point.
+ *   rmsmp_grouped_plan_bytes    scratch size for the table of these layers on the current device
+ *                               (the table proper plus N x K bytes per layer with PoT rows and
+ *                               without act_nonneg for the E4M3 copy of its activation codes, which
+ *                               every launch rewrites).
  *   rmsmp_gemm_grouped_prepare  validates the items, builds the table (tensor maps of every
  *                               layer's packed rows and activations, work lists per SM) and queues
  *                               its upload to d_table (256-byte aligned) on `stream`; fills *plan.
- *                               Every item needs N <= 128, else RMSMP_ERR_VARIANT.  The call costs
+ *                               Every item needs N <= 128, and K <= 16384 if it has PoT rows (the
+ *                               exactness bound of the fp32 sums), else RMSMP_ERR_VARIANT.  The call costs
  *                               host time proportional to the number of layers: do it once.
- *   rmsmp_gemm_grouped_launch   one kernel launch from a prepared plan; may be repeated for as
+ *   rmsmp_gemm_grouped_launch   one launch from a prepared plan (the streaming kernel, behind a small
+ *                               kernel that writes the activation copies); may be repeated for as
  *                               long as the buffers, shapes and leading dimensions the plan was
  *                               built from stay the same (their CONTENTS may change: new weights
  *                               packed with the same row map, new activation codes).  The table
@@ -302,7 +318,7 @@ typedef struct rmsmp_grouped_plan {
     int32_t grid;              /* CTAs of the launch */
     uint32_t smem_bytes;       /* dynamic shared memory per CTA */
     int32_t device;            /* ordinal of the device the table was built for */
-    int32_t reserved;
+    int32_t conv_grid;         /* blocks per layer of the kernel that writes the E4M3 activation copies (0: no PoT rows) */
     const void* d_table;
     uint64_t table_bytes;
 } rmsmp_grouped_plan;

@@ -58,14 +58,14 @@ class rmsmp_gemm_item(C.Structure):
     _fields_ = [
         ("layer", C.POINTER(rmsmp_layer)), ("d_packed", C.c_void_p), ("d_act", C.c_void_p),
         ("N", C.c_int64), ("ld_act", C.c_int64), ("act_step", C.c_float),
-        ("d_out", C.c_void_p), ("ld_out", C.c_int64), ("d_acc", C.c_void_p),
+        ("d_out", C.c_void_p), ("ld_out", C.c_int64), ("d_acc", C.c_void_p), ("act_nonneg", C.c_int32),
     ]
 
 
 class rmsmp_grouped_plan(C.Structure):
     _fields_ = [
         ("magic", C.c_uint32), ("count", C.c_int32), ("grid", C.c_int32), ("smem_bytes", C.c_uint32),
-        ("device", C.c_int32), ("reserved", C.c_int32), ("d_table", C.c_void_p), ("table_bytes", C.c_uint64),
+        ("device", C.c_int32), ("conv_grid", C.c_int32), ("d_table", C.c_void_p), ("table_bytes", C.c_uint64),
     ]
 
 
@@ -311,11 +311,13 @@ def rmsmp_grouped_table_bytes(count: int) -> int:
 
 
 def make_gemm_items(items):
-    """items: iterable of (layer, d_packed, d_act, N, ld_act, act_step, d_out, ld_out, d_acc|None)
+    """items: iterable of (layer, d_packed, d_act, N, ld_act, act_step, d_out, ld_out, d_acc|None[, act_nonneg])
     -> ctypes array of rmsmp_gemm_item (keep the layers alive while it is in use)."""
     items = list(items)
     arr = (rmsmp_gemm_item * len(items))()
-    for k, (layer, pk, act, N, ld_act, step, out, ld_out, acc) in enumerate(items):
+    for k, item in enumerate(items):
+        layer, pk, act, N, ld_act, step, out, ld_out, acc = item[:9]
+        arr[k].act_nonneg = int(item[9]) if len(item) > 9 else 0
         arr[k].layer = C.pointer(layer)
         arr[k].d_packed = pk.data_ptr(); arr[k].d_act = act.data_ptr()
         arr[k].N = N; arr[k].ld_act = ld_act; arr[k].act_step = step

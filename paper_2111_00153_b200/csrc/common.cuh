@@ -43,6 +43,7 @@ struct Problem {
     int B, H, W, Ho, Wo, stride, pad;
     int64_t pix_pitch;
     int64_t N;                // B*Ho*Wo
+    int act_nonneg;           // grouped tensor-core launch: every activation code is within 0..15
     // outputs
     float act_step;
     float* out;
@@ -109,11 +110,12 @@ cudaError_t launch_grouped(const uint8_t* d_table, size_t table_bytes, int64_t t
 // grouped tensor-core launch (stream.cu): table size, per-problem support test, host-side table and
 // launch geometry, launch
 int64_t stream_items_of(int nP, int nF4, int n8);
-size_t stream_table_bytes(int count, int64_t nitems, int sms);
+int64_t stream_act_bytes(int nP, int act_nonneg, int64_t N, int Kp);
+size_t stream_table_bytes(int count, int64_t nitems, int sms, int64_t act_bytes);
 bool stream_supported(const Problem& p);
 bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_table, size_t table_bytes,
-                        int* grid_out, uint32_t* smem_out);
-cudaError_t launch_stream(const uint8_t* d_table, int grid, uint32_t smem_bytes, cudaStream_t st);
+                        uint8_t* d_table, int* grid_out, uint32_t* smem_out, uint32_t* conv_grid_out);
+cudaError_t launch_stream(const uint8_t* d_table, int grid, uint32_t smem_bytes, int count, uint32_t conv_grid_x, cudaStream_t st);
 // returns false if the tensor variant cannot run this problem (alignment / shape)
 bool tensor_supported(const Problem& p);
 rmsmp_status launch_tensor(const Problem& p, cudaStream_t st);

@@ -550,6 +550,7 @@ static rmsmp_status grouped_problems(const rmsmp_gemm_item* h_items, int count, 
         p.pix_pitch = it.ld_act; p.N = it.N;
         p.act_step = it.act_step; p.out = it.d_out; p.acc = it.d_acc; p.ld_out = it.ld_out;
         p.out_mn = (out_layout == RMSMP_OUT_MN);
+        p.act_nonneg = it.act_nonneg != 0;
     }
     return RMSMP_OK;
 }
@@ -590,6 +591,15 @@ static int64_t grouped_row_blocks(const rmsmp_gemm_item* h_items, int count)
     return n;
 }
 
+// scratch of the E4M3 activation copies of the layers with PoT rows
+static int64_t grouped_act_bytes(const rmsmp_gemm_item* h_items, int count)
+{
+    int64_t n = 0;
+    for (int i = 0; i < count; ++i)
+        if (h_items[i].layer && h_items[i].N > 0) n += stream_act_bytes(h_items[i].layer->nP, h_items[i].act_nonneg, h_items[i].N, h_items[i].layer->Kp);
+    return n;
+}
+
 rmsmp_status rmsmp_grouped_plan_bytes(const rmsmp_gemm_item* h_items, int count, size_t* bytes)
 {
     if (!h_items || !bytes) return RMSMP_ERR_NULL;
@@ -600,7 +610,7 @@ rmsmp_status rmsmp_grouped_plan_bytes(const rmsmp_gemm_item* h_items, int count,
     }
     rmsmp_status a = check_arch();
     if (a != RMSMP_OK) return a;
-    *bytes = stream_table_bytes(count, grouped_row_blocks(h_items, count), sm_count());
+    *bytes = stream_table_bytes(count, grouped_row_blocks(h_items, count), sm_count(), grouped_act_bytes(h_items, count));
     return RMSMP_OK;
 }
 
@@ -617,15 +627,16 @@ rmsmp_status rmsmp_gemm_grouped_prepare(const rmsmp_gemm_item* h_items, int coun
     if (a != RMSMP_OK) return a;
     for (const Problem& p : probs)
         if (!stream_supported(p)) return RMSMP_ERR_VARIANT;
-    const size_t need = stream_table_bytes(count, grouped_row_blocks(h_items, count), sm_count());
+    const size_t need = stream_table_bytes(count, grouped_row_blocks(h_items, count), sm_count(), grouped_act_bytes(h_items, count));
     if (table_bytes < need) return RMSMP_ERR_BUFFER_TOO_SMALL;
-    std::vector<uint8_t> table(need);
+    const size_t head = stream_table_bytes(count, grouped_row_blocks(h_items, count), sm_count(), 0);      // the part the host fills
+    std::vector<uint8_t> table(head);
     int grid = 0;
-    uint32_t smem = 0;
-    if (!stream_build_table(probs.data(), count, sm_count(), table.data(), need, &grid, &smem)) return RMSMP_ERR_VARIANT;
+    uint32_t smem = 0, conv_grid = 0;
+    if (!stream_build_table(probs.data(), count, sm_count(), table.data(), need, static_cast<uint8_t*>(d_table), &grid, &smem, &conv_grid)) return RMSMP_ERR_VARIANT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the table leaves from pageable memory: the copy has read it when the call returns
-    if (cudaMemcpyAsync(d_table, table.data(), need, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    if (cudaMemcpyAsync(d_table, table.data(), head, cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return RMSMP_ERR_CUDA;
     }
@@ -633,6 +644,7 @@ rmsmp_status rmsmp_gemm_grouped_prepare(const rmsmp_gemm_item* h_items, int coun
     plan->count = count;
     plan->grid = grid;
     plan->smem_bytes = smem;
+    plan->conv_grid = (int32_t)conv_grid;
     plan->device = device_ordinal();
     plan->d_table = d_table;
     plan->table_bytes = need;
@@ -646,8 +658,9 @@ rmsmp_status rmsmp_gemm_grouped_launch(const rmsmp_grouped_plan* plan, void* str
     rmsmp_status a = check_arch();
     if (a != RMSMP_OK) return a;
     if (plan->device != device_ordinal()) return RMSMP_ERR_BAD_LAYER;
-    if (launch_stream(static_cast<const uint8_t*>(plan->d_table), plan->grid, plan->smem_bytes,
-                      static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    if (plan->conv_grid < 0 || plan->conv_grid > 65535) return RMSMP_ERR_BAD_LAYER;
+    if (launch_stream(static_cast<const uint8_t*>(plan->d_table), plan->grid, plan->smem_bytes, plan->count,
+                      (uint32_t)plan->conv_grid, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         cudaGetLastError();
         return RMSMP_ERR_CUDA;
     }

@@ -20,8 +20,15 @@
 //   warp 1       producer of the activation codes: per k-block one swizzled box [n_pad tokens][128
 //                codes] (rows beyond a layer's token count read zeros) into a ring of its own.
 //   warps 2-3    idle (they keep the warp numbering of the roles below a multiple of four).
-//   warps 4-7    MMA issuers.  tcgen05.mma kind::i8, M = 128 rows, N = n_pad tokens, A from tensor
-//                memory, B from shared memory, one instruction per 32 codes.  One thread gets an
+//   warps 4-7    MMA issuers.  tcgen05.mma, M = 128 rows, N = n_pad tokens, A from tensor memory, B
+//                from shared memory, one instruction per 32 codes.  Fixed-4 and Fixed-8 tiles are
+//                kind::i8 with int32 sums.  PoT-4 tiles are kind::f8f6f4: the code shifted left by two
+//                is a 6-bit float (E3M2) of a quarter of its value, the activations are E4M3 bytes, the
+//                sums are fp32 and exact (multiples of 1/4 below 2^22).  Activation bytes known to be
+//                within 0..15 are read as they are (as an E4M3 number such a byte is the code times
+//                2^-9, subnormals included); otherwise the E4M3 copy of a layer's codes is written
+//                once per launch by a small kernel in front of this one (act_e4m3_kernel, into
+//                scratch behind the table).  One thread gets an
 //                MMA out only every ~150 cycles whatever its size (measured; two issuing threads
 //                give twice the rate), so with few tokens the steps of a stage are dealt to up to
 //                four issuers, each with an accumulator chain of its own (the chains are added up
@@ -33,7 +40,7 @@
 //                the stage's 32-code steps.  Consecutive lanes read consecutive rows of the
 //                swizzled box (no bank conflicts).  16-byte raw chunk -> 32 int8 values in
 //                registers -> tcgen05.st into the stage's columns.
-//   warps 24-27  epilogue: tcgen05.ld, add the chains, undo the x16 of Fixed-4 rows, scale by
+//   warps 24-27  epilogue: tcgen05.ld, add the chains, undo the x16 of Fixed-4 rows (the 1/4 of PoT rows), scale by
 //                wstep * act_step, and store each lane's value to its ORIGINAL row.
 // Tensor memory: two accumulator buffers of nch * n_pad columns, then four to six A stages of 64 columns.
 // The epilogue looks one item ahead for its rows' permutation entries and scales, which live in
@@ -64,6 +71,7 @@ constexpr int kStreamThreads = 32 * (kProdWarps + kMmaWarps + kExpWarps + kEpiWa
 constexpr int kAStageCols = 64;                                       // 256 codes = 64 32-bit columns per lane
 constexpr int kMaxTokens = 128;                                       // accumulator columns of one chain at most
 constexpr int kRingMax = 12;
+constexpr int kStreamMaxK = 16384;                                    // reduction length up to which the fp32 sums of PoT tiles are exact
 constexpr int kLocalItems = 96;                                        // items of a CTA's list kept in shared memory
 constexpr int kStreamSmem = 232448 - 1024 - kLocalItems * 32;
 constexpr uint32_t kPlanMagic = 0x53545247u;                          // "STRG"
@@ -73,6 +81,11 @@ constexpr uint32_t kPlanMagic = 0x53545247u;                          // "STRG"
 struct alignas(128) StreamProblem {
     CUtensorMap q4[3], q8[3];       // packed 4-bit / 8-bit rows; boxes of 128, 64 and 32 rows x 128 bytes
     CUtensorMap act;                // activation codes [N][ld_act]; box n_pad tokens x 128 codes
+    CUtensorMap act_fp;             // what the PoT tiles read: the E4M3 copy [N][Kp], or the codes themselves (act_nonneg)
+    const int8_t* act_src;          // the codes, and where the copy goes (nullptr: no PoT rows)
+    uint8_t* act_fp_dst;
+    int64_t pix_pitch;
+    int32_t Cin, Kp;
     const int32_t* perm;
     const float* wstep;
     float* out;
@@ -81,7 +94,7 @@ struct alignas(128) StreamProblem {
     int64_t ld_out;
     float act_step;
     int32_t M, N, nkb, out_mn;
-    int32_t pad0[13];
+    float fp_unit;                  // integer sum = fp32 sum of a PoT tile x this: 4 with the copy, 2^11 with raw bytes (code x 2^-9)
 };
 static_assert(sizeof(StreamProblem) % 128 == 0, "tensor maps stay 128-byte aligned in the array");
 
@@ -96,7 +109,10 @@ struct StreamHeader {               // first 128 bytes of the table
     uint32_t stage_bytes, b_bytes, idesc, smem_bytes;   // one slot of the packed-code ring / of the activation ring
     int32_t acc_cols, nAst;                   // tensor memory: columns of one accumulator buffer (nch * n_pad); A stages behind the two buffers
     uint32_t off_first, off_items, off_probs, bytes;
-    uint32_t pad[14];
+    uint32_t idesc_fp;                        // instruction descriptor of PoT tiles (E3M2 x E4M3 -> fp32)
+    uint32_t off_act, n_fp;                   // scratch of the E4M3 activation copies; layers that have one
+    uint32_t conv_grid_x;                     // blocks per layer of the kernel that writes them
+    uint32_t pad[10];
 };
 static_assert(sizeof(StreamHeader) == 128, "header is 128 bytes");
 
@@ -105,6 +121,40 @@ __host__ __device__ inline int box_index(int rows) { return rows > 64 ? 0 : (row
 __device__ __forceinline__ void lds128(uint32_t addr, uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d)
 {
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr) : "memory");
+}
+
+// A PoT-4 code (sign << 3 | e, value +-2^(e-1), e = 0: zero; Eq. 4) shifted left by two IS the 6-bit
+// float with three exponent and two mantissa bits (bias 3, mantissa 00, exponent field 0 = zero) of a
+// quarter of that value.  The tensor core takes such numbers in 8-bit containers (kind::f8f6f4, A format
+// E3M2), multiplies exactly and adds in fp32, which is exact here: every product and every partial sum is
+// a multiple of one unit (1/4, or 2^-11 with activation bytes read as they are) below 2^24 units (the host
+// checks the reduction length).  So PoT rows need no table: two shifts and two masks spread the even and
+// the odd codes of a word over two words, and two byte permutes put them back in order.
+__device__ __forceinline__ void expand_pot_chunk_e3m2(const uint4& c, uint32_t out[8])
+{
+    const uint32_t x[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t ev = (x[i] << 2) & 0x3C3C3C3Cu, od = (x[i] >> 2) & 0x3C3C3C3Cu;
+        out[2 * i] = prmt(ev, od, 0x5140u);
+        out[2 * i + 1] = prmt(ev, od, 0x7362u);
+    }
+}
+
+// Four int8 activation codes (each within -16..16) as four E4M3 bytes, exactly: byte + 128 is put under
+// the fp16 exponent of 1024, 1152 is subtracted, and the pair is narrowed by the hardware conversion.
+__device__ __forceinline__ uint32_t e4m3x4_of_s8x4(uint32_t w)
+{
+    const uint32_t u = w ^ 0x80808080u;
+    uint32_t h01 = prmt(u, 0x64646464u, 0x5140u), h23 = prmt(u, 0x64646464u, 0x7362u), d;
+    asm("{\n\t.reg .b16 lo, hi;\n\t"
+        "sub.rn.f16x2 %1, %1, %3;\n\t"
+        "sub.rn.f16x2 %2, %2, %3;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f16x2 lo, %1;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f16x2 hi, %2;\n\t"
+        "mov.b32 %0, {lo, hi};\n\t}"
+        : "=r"(d), "+r"(h01), "+r"(h23) : "r"(0x64806480u));
+    return d;
 }
 
 // 32-byte piece `g` (0..3) of this thread's 128-byte raw row, expanded to 16 words of int8 values:
@@ -121,7 +171,7 @@ __device__ __forceinline__ void stream_expand(int kind, uint32_t row, uint32_t p
         return;
     }
     uint32_t lo[8], hi[8];
-    if (kind == kPoT4) { expand_pot_chunk(c0, lo); expand_pot_chunk(c1, hi); }
+    if (kind == kPoT4) { expand_pot_chunk_e3m2(c0, lo); expand_pot_chunk_e3m2(c1, hi); }
     else { expand_fixed4_chunk_x16(c0, lo); expand_fixed4_chunk_x16(c1, hi); }
 #pragma unroll
     for (int t = 0; t < 8; ++t) { w[t] = lo[t]; w[8 + t] = hi[t]; }
@@ -171,21 +221,71 @@ __device__ __forceinline__ void mma_i8_tmem_a(uint32_t d_tmem, uint32_t a_tmem, 
         : "memory");
 }
 
+// The same with E3M2 x E4M3 operands and fp32 accumulators.
+__device__ __forceinline__ void mma_f8f6f4_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                                  uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // The tensor maps live in the table in global memory (written by a copy before the launch); fetching a
 // tile's descriptor one tile ahead keeps its first copy from waiting for it.
 __device__ __forceinline__ void tensormap_prefetch(const CUtensorMap* m)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");
 }
+// E4M3 copies of the activation codes of every layer with PoT rows: [N][Kp], zeros beyond the layer's
+// reduction length.  blockIdx.y = layer; layers whose bytes can be read as they are have no copy.
+__global__ void __launch_bounds__(256) act_e4m3_kernel(const uint8_t* __restrict__ table)
+{
+    // Programmatic dependent launch on both sides: the streaming kernel behind this one may start at once, and
+    // this kernel may have started before the launch in front of it (which may still read the copies) is over.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const StreamHeader* H = reinterpret_cast<const StreamHeader*>(table);
+    const StreamProblem& P = reinterpret_cast<const StreamProblem*>(table + H->off_probs)[blockIdx.y];
+    if (!P.act_fp_dst) return;
+    const int upr = P.Kp >> 4;                            // 16-byte units per row
+    const int units = P.N * upr;
+    for (int u = blockIdx.x * 256 + threadIdx.x; u < units; u += gridDim.x * 256) {
+        const int n = u / upr, k0 = (u - n * upr) << 4;
+        const int8_t* src = P.act_src + (int64_t)n * P.pix_pitch + k0;
+        uint4 v;
+        if (k0 + 16 <= P.Cin) {
+            v = *reinterpret_cast<const uint4*>(src);
+        } else {
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+            for (int b = 0; b < 16 && k0 + b < P.Cin; ++b) w[b >> 2] |= (uint32_t)(uint8_t)src[b] << (8 * (b & 3));
+            v = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        uint4 o;
+        o.x = e4m3x4_of_s8x4(v.x); o.y = e4m3x4_of_s8x4(v.y);
+        o.z = e4m3x4_of_s8x4(v.z); o.w = e4m3x4_of_s8x4(v.w);
+        *reinterpret_cast<uint4*>(P.act_fp_dst + (int64_t)n * P.Kp + k0) = o;
+    }
+}
+
 __global__ void __launch_bounds__(kStreamThreads, 1)
 stream_kernel(const uint8_t* __restrict__ table)
 {
+    // The next launch on the stream may start while this one runs (programmatic dependent launch): its CTAs
+    // take the SMs this launch's CTAs leave.  In turn this kernel may run beside the launch in front of it, so
+    // what that launch may still read or write is touched only behind griddepcontrol.wait: the activation
+    // copies (activation producer) and the outputs (epilogue).  Both roles exist in every CTA, so no CTA, and
+    // hence no launch, ends before the launch in front of it has.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const StreamHeader* H = reinterpret_cast<const StreamHeader*>(table);
     const int32_t* cta_first = reinterpret_cast<const int32_t*>(table + H->off_first);
     const StreamItem* items = reinterpret_cast<const StreamItem*>(table + H->off_items);
     const StreamProblem* probs = reinterpret_cast<const StreamProblem*>(table + H->off_probs);
     const int n_pad = H->n_pad, nS = H->nS, nch = H->nch, nB = H->nB, nAst = H->nAst;
-    const uint32_t stage_bytes = H->stage_bytes, b_bytes = H->b_bytes, idesc = H->idesc;
+    const uint32_t stage_bytes = H->stage_bytes, b_bytes = H->b_bytes, idesc = H->idesc, idesc_fp = H->idesc_fp;
     const uint32_t acc_cols = (uint32_t)H->acc_cols, a_base_col = 2u * acc_cols;
     const uint32_t b_sub = (uint32_t)n_pad * 128u;
 
@@ -294,10 +394,13 @@ stream_kernel(const uint8_t* __restrict__ table)
         // ---------------------------------------------------------- producer of the activation tiles (lanes 0 / 1: first / second k-block)
         uint32_t sb = 0, phB = 0;
         bool ok = true;
+        // the E4M3 copies come from the kernel in front of this one
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         for (int it = it0; it < it1 && ok; ++it) {
             const ItemView v = view(it);
             last_status = v.P->status;
-            if (lane == 0 && it + 1 < it1) tensormap_prefetch(&view(it + 1).P->act);
+            const CUtensorMap* amap = (v.kind == kPoT4) ? &v.P->act_fp : &v.P->act;
+            if (lane == 0 && it + 1 < it1) { const ItemView nv = view(it + 1); tensormap_prefetch(nv.kind == kPoT4 ? &nv.P->act_fp : &nv.P->act); }
             for (int st = 0; st < v.nst; ++st) {
                 if (!mbar_wait_parked_warp(bar_emptyA + 8 * sb, phB ^ 1, abort_flag)) { ok = false; break; }    // activation slot s goes with A stage s
                 const uint32_t fbar = bar_fullB + 8 * sb;
@@ -305,7 +408,7 @@ stream_kernel(const uint8_t* __restrict__ table)
                 const int nsub = min(v.kbps, v.nkb - kb0);
                 if (lane == 0) mbar_arrive_expect_tx(fbar, (uint32_t)nsub * b_sub);
                 __syncwarp();
-                if (lane < nsub) tma_load_2d(sB + sb * b_bytes + (uint32_t)lane * b_sub, &v.P->act, fbar, (kb0 + lane) * 128, 0);
+                if (lane < nsub) tma_load_2d(sB + sb * b_bytes + (uint32_t)lane * b_sub, amap, fbar, (kb0 + lane) * 128, 0);
                 if (++sb == (uint32_t)nAst) { sb = 0; phB ^= 1; }
             }
         }
@@ -346,9 +449,16 @@ stream_kernel(const uint8_t* __restrict__ table)
                             // a 32-code step is 8 columns of A and 32 bytes (two 16-byte units) of a B row; the first
                             // instruction into a chain in this item overwrites it
                             const int nsteps = 4 * min(v.kbps, v.nkb - st * v.kbps);
-                            for (int j = 0; j < nsteps; ++j) {
-                                const uint32_t b_j = b_lo + (uint32_t)(j >> 2) * (b_sub >> 4) + 2u * (uint32_t)(j & 3);
-                                mma_i8_tmem_a(d_tmem, a_t + 8 * j, b_j, desc_hi, idesc, (st < nch && j == 0) ? 0u : 1u);
+                            if (v.kind == kPoT4) {
+                                for (int j = 0; j < nsteps; ++j) {
+                                    const uint32_t b_j = b_lo + (uint32_t)(j >> 2) * (b_sub >> 4) + 2u * (uint32_t)(j & 3);
+                                    mma_f8f6f4_tmem_a(d_tmem, a_t + 8 * j, b_j, desc_hi, idesc_fp, (st < nch && j == 0) ? 0u : 1u);
+                                }
+                            } else {
+                                for (int j = 0; j < nsteps; ++j) {
+                                    const uint32_t b_j = b_lo + (uint32_t)(j >> 2) * (b_sub >> 4) + 2u * (uint32_t)(j & 3);
+                                    mma_i8_tmem_a(d_tmem, a_t + 8 * j, b_j, desc_hi, idesc, (st < nch && j == 0) ? 0u : 1u);
+                                }
                             }
                             mma_commit(bar_emptyA + 8 * sa);
                         }
@@ -436,6 +546,7 @@ stream_kernel(const uint8_t* __restrict__ table)
         };
         float scale, scale_n; int shift, shift_n, m, m_n;
         row_info(it0, scale, shift, m);
+        asm volatile("griddepcontrol.wait;" ::: "memory");      // the launch in front of this one may still be writing the same outputs
         for (int it = it0; it < it1 && alive; ++it, ++n) {
             const ItemView vi = view(it);
             const StreamProblem* P = vi.P;
@@ -466,14 +577,25 @@ stream_kernel(const uint8_t* __restrict__ table)
             };
             // 16 tokens at a time; with few tokens the 32-code steps went to nch accumulator chains in turn: add them
             const int n16 = (N + 15) >> 4;
+            const bool fp = vi.kind == kPoT4;            // fp32 sums: add the chains (exactly), then the integer number of units
+            const float fp_unit = P->fp_unit;
             for (int ch = 0; ch < n16; ++ch) {
                 uint32_t v[16];
                 tmem_ld16(taddr + ch * 16, v);
                 for (int c = 1; c < nchains; ++c) {
                     uint32_t u[16];
                     tmem_ld16(taddr + c * n_pad + ch * 16, u);
+                    if (fp) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] += u[j];
+                        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__fadd_rn(__uint_as_float(v[j]), __uint_as_float(u[j])));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] += u[j];
+                    }
+                }
+                if (fp) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__float2int_rn(__fmul_rn(__uint_as_float(v[j]), fp_unit));
                 }
                 if (ch == n16 - 1) release_tmem();
                 if (m < 0) continue;
@@ -502,7 +624,7 @@ inline size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
     int grid, nitems;
-    size_t off_first, off_items, off_probs, bytes;
+    size_t off_first, off_items, off_probs, off_act, bytes;      // bytes: the table proper; the E4M3 copies follow at off_act
 };
 
 Layout table_layout(int count, int nitems, int grid)
@@ -514,6 +636,7 @@ Layout table_layout(int count, int nitems, int grid)
     L.off_items = off; off = up(off + sizeof(StreamItem) * (size_t)nitems, 128);
     L.off_probs = off; off += sizeof(StreamProblem) * (size_t)count;
     L.bytes = up(off, 256);
+    L.off_act = L.bytes;
     return L;
 }
 
@@ -526,9 +649,15 @@ int64_t stream_items_of(int nP, int nF4, int n8)
 }
 
 // Scratch bytes the table of `count` layers with `nitems` tiles needs on a device with `sms` SMs.
-size_t stream_table_bytes(int count, int64_t nitems, int sms)
+size_t stream_table_bytes(int count, int64_t nitems, int sms, int64_t act_bytes)
 {
-    return table_layout(count, (int)nitems, sms).bytes;
+    return table_layout(count, (int)nitems, sms).bytes + (size_t)act_bytes;
+}
+
+// Bytes of the E4M3 activation copy of one layer (0 without PoT rows).
+int64_t stream_act_bytes(int nP, int act_nonneg, int64_t N, int Kp)
+{
+    return (nP > 0 && !act_nonneg) ? (int64_t)up((size_t)(N * Kp), 256) : 0;
 }
 
 // Can this problem be part of a grouped tensor-core launch?
@@ -536,13 +665,15 @@ bool stream_supported(const Problem& p)
 {
     if (p.kh != 1 || p.kw != 1 || p.N < 1 || p.N > kMaxTokens) return false;
     if (p.pix_pitch % 16 != 0 || (reinterpret_cast<uintptr_t>(p.act) & 15) != 0) return false;
+    // PoT tiles are summed in fp32 in units of 1/4: exact while 64 * 16 * K <= 2^24
+    if (p.nP > 0 && p.Kp > kStreamMaxK) return false;
     return tensor_map_encoder() != nullptr;
 }
 
 // Builds the table on the host (`h_table`, stream_table_bytes(...) bytes) and the launch geometry.
 // Returns false if a tensor map cannot be encoded or the shared-memory budget does not fit.
 bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_table, size_t table_bytes,
-                        int* grid_out, uint32_t* smem_out)
+                        uint8_t* d_table, int* grid_out, uint32_t* smem_out, uint32_t* conv_grid_out)
 {
     EncodeTiledFn enc = tensor_map_encoder();
     if (!enc) return false;
@@ -555,7 +686,9 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
     if (nitems >= (1ll << 30)) return false;
     const int grid = (int)std::min<int64_t>(sms, nitems);
     const Layout L = table_layout(count, (int)nitems, grid);
-    if (L.bytes > table_bytes) return false;
+    int64_t act_bytes = 0;
+    for (int i = 0; i < count; ++i) act_bytes += stream_act_bytes(probs[i].nP, probs[i].act_nonneg, probs[i].N, probs[i].Kp);
+    if (L.bytes + (size_t)act_bytes > table_bytes) return false;
     memset(h_table, 0, L.bytes);
     StreamHeader* H = reinterpret_cast<StreamHeader*>(h_table);
     H->magic = kPlanMagic; H->nprob = count; H->nitems = (int32_t)nitems; H->grid = grid;
@@ -578,11 +711,16 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
     H->smem_bytes = (uint32_t)(H->nB * H->b_bytes + H->nS * H->stage_bytes + 1024 + 64 * kRingMax);
     // kind::i8: int32 accumulate, signed 8-bit A and B, both K-major, N/8 at bit 17, M/16 at bit 24
     H->idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(H->n_pad >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
+    // kind::f8f6f4: fp32 accumulate (1 at bit 4), A = E3M2 (4 at bit 7), B = E4M3 (0 at bit 10)
+    H->idesc_fp = (1u << 4) | (4u << 7) | (0u << 10) | ((uint32_t)(H->n_pad >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
     H->off_first = (uint32_t)L.off_first; H->off_items = (uint32_t)L.off_items; H->off_probs = (uint32_t)L.off_probs;
     H->bytes = (uint32_t)L.bytes;
+    H->off_act = (uint32_t)L.off_act;
 
     // problems and their tensor maps
     StreamProblem* sp = reinterpret_cast<StreamProblem*>(h_table + L.off_probs);
+    size_t act_off = 0;
+    int64_t max_units = 0;
     for (int i = 0; i < count; ++i) {
         const Problem& p = probs[i];
         StreamProblem& q = sp[i];
@@ -609,11 +747,32 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
                 return false;
         }
+        q.fp_unit = p.act_nonneg ? 2048.0f : 4.0f;
+        if (p.nP > 0 && p.act_nonneg) {
+            q.act_fp = q.act;
+        } else if (p.nP > 0) {
+            q.act_src = p.act;
+            q.act_fp_dst = d_table + L.off_act + act_off;
+            q.pix_pitch = p.pix_pitch; q.Cin = p.Cin; q.Kp = p.Kp;
+            act_off += (size_t)stream_act_bytes(p.nP, p.act_nonneg, p.N, p.Kp);
+            H->n_fp += 1;
+            max_units = std::max<int64_t>(max_units, p.N * (int64_t)(p.Kp / 16));
+            const cuuint64_t gd[2] = {(cuuint64_t)p.Kp, (cuuint64_t)p.N};
+            const cuuint64_t gs[1] = {(cuuint64_t)p.Kp};
+            const cuuint32_t bx[2] = {128u, (cuuint32_t)H->n_pad};
+            const cuuint32_t es[2] = {1, 1};
+            if (enc(&q.act_fp, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, q.act_fp_dst, gd, gs, bx, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return false;
+        }
         q.perm = p.perm; q.wstep = p.wstep;
         q.out = p.out; q.acc = p.acc; q.status = p.status; q.ld_out = p.ld_out;
         q.act_step = p.act_step; q.M = p.M; q.N = (int32_t)p.N;
         q.nkb = p.Kp / 128; q.out_mn = p.out_mn;
     }
+
+    H->conv_grid_x = (uint32_t)std::max<int64_t>(1, std::min<int64_t>(64, (max_units + 255) / 256));
 
     // work items: every tile of every layer, handed to the CTAs longest first onto the least loaded one; an
     // item's cost is the bytes it streams (in 128-byte rows) plus a constant for start-up and output
@@ -658,15 +817,29 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
     first[grid] = pos;
     *grid_out = grid;
     *smem_out = H->smem_bytes;
+    if (H->n_fp == 0) H->conv_grid_x = 0;
+    *conv_grid_out = H->conv_grid_x;
     return true;
 }
 
-cudaError_t launch_stream(const uint8_t* d_table, int grid, uint32_t smem_bytes, cudaStream_t st)
+// Both kernels are launched as programmatic dependents of whatever is in front of them on the stream.
+// conv_grid_x > 0: layers with PoT rows are part of the launch; their activation copies are written first.
+cudaError_t launch_stream(const uint8_t* d_table, int grid, uint32_t smem_bytes, int count, uint32_t conv_grid_x, cudaStream_t st)
 {
     static bool attr_set[kMaxDevices] = {};
     if (!ensure_smem_attr(reinterpret_cast<const void*>(stream_kernel), kStreamSmem, attr_set)) return cudaErrorUnknown;
-    stream_kernel<<<grid, kStreamThreads, smem_bytes, st>>>(d_table);
-    return cudaGetLastError();
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 1;
+    if (conv_grid_x != 0) {
+        cfg.gridDim = dim3(conv_grid_x, (unsigned)count); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, act_e4m3_kernel, d_table);
+        if (e != cudaSuccess) return e;
+    }
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(kStreamThreads); cfg.dynamicSmemBytes = smem_bytes;
+    return cudaLaunchKernelEx(&cfg, stream_kernel, d_table);
 }
 
 }  // namespace rmsmp

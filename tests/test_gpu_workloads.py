@@ -265,7 +265,8 @@ def _grouped_case(shapes, N, layout=R.OUT_NM):
         acc = torch.full(shape, -5, dtype=torch.int32, device="cuda") if i != 1 else None
         step = float(np.float32(0.01 * (i + 1)))
         keep.append((layer, d_packed, a, y, acc))
-        items.append((layer, d_packed, a, N, ld, step, y, shape[1], acc))
+        # unsigned codes: every other such layer says so (its bytes are then read as they are by the PoT tiles)
+        items.append((layer, d_packed, a, N, ld, step, y, shape[1], acc, 1 if i % 4 == 0 else 0))
         v_ref, wstep = O.quantize_rows(W, scheme, bits, alpha)
         acc_ref = O.matmul(v_ref, act)
         refs.append((acc_ref, _expected(acc_ref, wstep, np.float32(step))))
