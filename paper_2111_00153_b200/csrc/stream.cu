@@ -32,8 +32,8 @@
 //                MMA out only every ~150 cycles whatever its size (measured; two issuing threads
 //                give twice the rate), so with few tokens the steps of a stage are dealt to up to
 //                four issuers, each with an accumulator chain of its own (the chains are added up
-//                in the epilogue).  Warp 4 allocates tensor memory.  Accumulator buffers alternate
-//                between items so that an item's output overlaps the next item's stream.
+//                in the epilogue).  Warp 4 allocates tensor memory.  Accumulator buffers take turns
+//                between items so that an item's output overlaps the next items' stream.
 //   warps 8-23   expanders, in two sets that take alternate stages (one set's waits fall into the
 //                other's arithmetic).  A warp may touch the 32 tensor-memory lanes of its quarter
 //                (warp % 4); thread <-> one row of the tile; a quarter's two warps of a set split
@@ -42,7 +42,7 @@
 //                registers -> tcgen05.st into the stage's columns.
 //   warps 24-27  epilogue: tcgen05.ld, add the chains, undo the x16 of Fixed-4 rows (the 1/4 of PoT rows), scale by
 //                wstep * act_step, and store each lane's value to its ORIGINAL row.
-// Tensor memory: two accumulator buffers of nch * n_pad columns, then four to six A stages of 64 columns.
+// Tensor memory: two or four accumulator buffers of nch * n_pad columns, then four to six A stages of 64 columns.
 // The epilogue looks one item ahead for its rows' permutation entries and scales, which live in
 // each layer's packed buffer; everything else an item needs is in the table.
 // Every mbarrier wait is bounded; a wait that runs out sets the abort flag, all roles leave, tensor
@@ -112,7 +112,8 @@ struct StreamHeader {               // first 128 bytes of the table
     uint32_t idesc_fp;                        // instruction descriptor of PoT tiles (E3M2 x E4M3 -> fp32)
     uint32_t off_act, n_fp;                   // scratch of the E4M3 activation copies; layers that have one
     uint32_t conv_grid_x;                     // blocks per layer of the kernel that writes them
-    uint32_t pad[10];
+    int32_t nAcc;                             // accumulator buffers in tensor memory (2 or 4): items in flight between issuers and epilogue
+    uint32_t pad[9];
 };
 static_assert(sizeof(StreamHeader) == 128, "header is 128 bytes");
 
@@ -286,7 +287,7 @@ stream_kernel(const uint8_t* __restrict__ table)
     const StreamProblem* probs = reinterpret_cast<const StreamProblem*>(table + H->off_probs);
     const int n_pad = H->n_pad, nS = H->nS, nch = H->nch, nB = H->nB, nAst = H->nAst;
     const uint32_t stage_bytes = H->stage_bytes, b_bytes = H->b_bytes, idesc = H->idesc, idesc_fp = H->idesc_fp;
-    const uint32_t acc_cols = (uint32_t)H->acc_cols, a_base_col = 2u * acc_cols;
+    const uint32_t acc_cols = (uint32_t)H->acc_cols, nAcc = (uint32_t)H->nAcc, a_base_col = nAcc * acc_cols;
     const uint32_t b_sub = (uint32_t)n_pad * 128u;
 
     extern __shared__ uint8_t smem_raw[];
@@ -297,7 +298,7 @@ stream_kernel(const uint8_t* __restrict__ table)
     const uint32_t bar_fullA = sBar, bar_emptyA = sBar + 8 * kRingMax;
     const uint32_t bar_full = sBar + 16 * kRingMax, bar_empty = sBar + 24 * kRingMax;
     const uint32_t bar_fullB = sBar + 32 * kRingMax;
-    const uint32_t bar_tfull = sBar + 48 * kRingMax, bar_tempty = bar_tfull + 16;
+    const uint32_t bar_tfull = sBar + 48 * kRingMax, bar_tempty = bar_tfull + 32;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     struct LocalItem { int4 a; int nkb, pad[3]; };        // the table's item (prob, kind << 16 | rows, row0, packed0) and its layer's k-blocks
@@ -319,7 +320,7 @@ stream_kernel(const uint8_t* __restrict__ table)
             mbar_init(bar_empty + 8 * s, kExpWarps / 2); // the stage's expander warps, as soon as the codes are in their registers
             mbar_init(bar_fullB + 8 * s, 1);             // the activation producer (+ transaction bytes)
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < 4; ++b) {
             mbar_init(bar_tfull + 8 * b, nch);           // every issuer's tcgen05.commit
             mbar_init(bar_tempty + 8 * b, kEpiWarps);    // one arrival per epilogue warp
         }
@@ -432,12 +433,12 @@ stream_kernel(const uint8_t* __restrict__ table)
             for (int it = it0; it < it1 && ok && !*abort_flag; ++it, ++n) {
                 const ItemView v = view(it);
                 last_status = v.P->status;
-                const uint32_t ab = n & 1;
+                const uint32_t ab = n % nAcc, lap = n / nAcc;
                 bool have_acc = false;                    // this issuer has made sure the item's accumulator buffer is free
                 for (int st = 0; st < v.nst; ++st, ++t) {
                     if ((int)(t % (uint32_t)nch) == me) {
                         if (!have_acc) {
-                            if (!mbar_wait_parked(bar_tempty + 8 * ab, ((n >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                            if (!mbar_wait_parked(bar_tempty + 8 * ab, (lap & 1) ^ 1, abort_flag)) { ok = false; break; }
                             have_acc = true;
                         }
                         if (!mbar_wait_parked(bar_fullB + 8 * sa, phA, abort_flag) || !mbar_wait_parked(bar_fullA + 8 * sa, phA, abort_flag)) { ok = false; break; }
@@ -469,7 +470,7 @@ stream_kernel(const uint8_t* __restrict__ table)
                 // Every issuer reports once per item, whether or not a stage of it was its own.  An issuer without
                 // stages in short items can be items ahead of the others: before it reports on this buffer again
                 // it makes sure that the buffer's previous item has everybody's report (one arrival per phase).
-                if (n >= 2 && !mbar_wait_parked(bar_tfull + 8 * ab, ((n - 2) >> 1) & 1, abort_flag)) break;
+                if (lap >= 1 && !mbar_wait_parked(bar_tfull + 8 * ab, (lap - 1) & 1, abort_flag)) break;
                 if (issuer) mma_commit(bar_tfull + 8 * ab);
             }
         }
@@ -552,8 +553,8 @@ stream_kernel(const uint8_t* __restrict__ table)
             const StreamProblem* P = vi.P;
             last_status = P->status;
             row_info(it + 1, scale_n, shift_n, m_n);
-            const uint32_t ab = n & 1;
-            if (!mbar_wait_parked_warp(bar_tfull + 8 * ab, (n >> 1) & 1, abort_flag)) { alive = false; break; }
+            const uint32_t ab = n % nAcc;
+            if (!mbar_wait_parked_warp(bar_tfull + 8 * ab, (n / nAcc) & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * acc_cols;
             const int N = P->N;
@@ -697,7 +698,10 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
     // for several chains, one per issuing thread (summed in the epilogue)
     H->nch = H->n_pad <= 32 ? 4 : (H->n_pad <= 64 ? 2 : 1);
     H->acc_cols = H->nch * H->n_pad;                              // <= 128
-    H->nAst = std::min(6, (512 - 2 * H->acc_cols) / kAStageCols) & ~1;      // even: the two expander sets alternate
+    // a short item's output (tensor-memory loads, scattered stores) takes about as long as its stream: with four
+    // accumulator buffers the issuers do not wait for it
+    H->nAcc = H->acc_cols <= 64 ? 4 : 2;
+    H->nAst = std::min(6, (512 - H->nAcc * H->acc_cols) / kAStageCols) & ~1;      // even: the two expander sets alternate
     H->b_bytes = (uint32_t)(2 * H->n_pad * 128);
     H->stage_bytes = 128u * 128u;                                 // one box: at most 128 rows x 128 bytes
     // Shared memory: a packed-code slot is held from the moment its copy is started until the expanders have the
@@ -775,7 +779,7 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
     H->conv_grid_x = (uint32_t)std::max<int64_t>(1, std::min<int64_t>(64, (max_units + 255) / 256));
 
     // work items: every tile of every layer, handed to the CTAs longest first onto the least loaded one; an
-    // item's cost is the bytes it streams (in 128-byte rows) plus a constant for start-up and output
+    // item's cost is its stages, weighted by kind and box height, plus a constant for start-up and output
     struct Cand { int64_t cost; StreamItem item; };
     std::vector<Cand> cand;
     cand.reserve((size_t)nitems);
@@ -789,7 +793,10 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
             for (int r = 0; r < n_of[k]; r += 128) {
                 const int rows = std::min(128, n_of[k] - r);
                 const int nst = (k == kFixed8) ? nkb : (nkb + 1) / 2;
-                const int64_t cost = (int64_t)nst * (128 >> box_index(rows)) + 96;
+                // measured: a stage of a full PoT / Fixed-4 / Fixed-8 tile takes about 1.11 : 1 : 0.79, half of it whatever
+                // the height of its box; an item's start-up and output about 3/4 of a full stage
+                static const int kind_weight[3] = {111, 100, 79};
+                const int64_t cost = (int64_t)nst * kind_weight[k] * (64 + (64 >> box_index(rows))) + 9600;
                 cand.push_back({cost, {i, (k << 16) | rows, region_row0[k] + r, perm0[k] + r}});
             }
     }
