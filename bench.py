@@ -566,15 +566,20 @@ def weights_leg(R, torch, peaks, tokens=(1, 8, 128), reps=5, launches=20, warm=5
     prepared once; a pass is one launch; `launches` passes run back to back between two events."""
     stack = bert_large_stack(R, torch)
     rows = []
-    for N in tokens:
+    # unsigned codes (Eq. 1) at every token count, read as they are by the PoT tiles; one more row with signed
+    # codes, which go through the E4M3 copy
+    for N, signed in [(n, False) for n in tokens] + [(8, True)]:
         keep, items, alg, wbytes, ops = [], [], 0, 0, 0
-        g = synth.rng(5, 9000 + N)
+        g = synth.rng(5, 9000 + N + (500 if signed else 0))
         for lay, pk in stack:
             M, K = lay.M, lay.Cin
-            act = torch.from_numpy(synth.act_codes_uniform(g, (N, K))).cuda()
+            codes = synth.act_codes_uniform(g, (N, K))
+            if signed:
+                codes = (codes.astype(np.int16) - 8).astype(np.int8)
+            act = torch.from_numpy(codes).cuda()
             y = torch.empty((N, M), dtype=torch.float32, device="cuda")
             keep.append((act, y))
-            items.append((lay, pk, act, N, K, 0.1, y, M, None, 1))      # codes 0..15: act_nonneg
+            items.append((lay, pk, act, N, K, 0.1, y, M, None, 0 if signed else 1))
             w = (lay.nP + lay.nF4) * K // 2 + lay.n8 * K + 8 * M
             wbytes += w
             alg += w + N * K + 4 * N * M
@@ -597,7 +602,7 @@ def weights_leg(R, torch, peaks, tokens=(1, 8, 128), reps=5, launches=20, warm=5
         ms = float(np.median(best))
         for lay, pk in stack[:3]:
             assert R.rmsmp_last_device_status(pk) == R.OK
-        rows.append({"tokens": N, "us": ms * 1e3, "gbs": alg / (ms * 1e-3) / 1e9, "frac": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        rows.append({"tokens": N, "codes": "signed (E4M3 copy per launch)" if signed else "unsigned (act_nonneg)", "us": ms * 1e3, "gbs": alg / (ms * 1e-3) / 1e9, "frac": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                      "tops": ops / (ms * 1e-3) / 1e12, "algorithmic_bytes": float(alg), "packed_weight_bytes": float(wbytes)})
         del keep, items, arr, table, plan
     head = rows[min(1, len(rows) - 1)]                    # the N = 8 row speaks for the regime
