@@ -557,6 +557,28 @@ def second_workloads_leg(R, torch, peaks, i8_peak):
         real_cin = 3 if k == 7 else Cin
         record(name + " B=%d" % B, lay, ms, 2 * M * real_cin * k * k * N,
                (lay.nP + lay.nF4) * real_cin * k * k // 2 + lay.n8 * real_cin * k * k + 8 * M + B * H * H * real_cin + 4 * N * M)
+    # the same first layer with its three channels as they are: patch matrix (rmsmp_im2col_codes), then the layer as
+    # a linear layer over the patches (K = 147 padded to 160); the step is both kernels
+    M, Cin, k, stride, pad, H = 64, 3, 7, 2, 3, 224
+    W = synth.weights_kaiming(synth.rng(7, M + 16 + k), M, 16, k, k)[:, :3]
+    K, ld = k * k * Cin, (k * k * Cin + 15) // 16 * 16
+    Wl = np.zeros((M, ld, 1, 1), np.float32)
+    Wl[:, :K, 0, 0] = W.transpose(0, 2, 3, 1).reshape(M, K)
+    lay, pk = pack(Wl)
+    ws = torch.empty(R.rmsmp_workspace_bytes(lay), dtype=torch.int8, device="cuda")
+    R.rmsmp_expand_weights(lay, pk, ws)
+    Ho = (H + 2 * pad - k) // stride + 1
+    N = B * Ho * Ho
+    act = torch.randint(0, 16, (B, H, H, Cin), dtype=torch.int8, device="cuda")
+    cols = torch.empty((N, ld), dtype=torch.int8, device="cuda")
+    y = torch.empty((N, M), dtype=torch.float32, device="cuda")
+
+    def first_layer():
+        R.rmsmp_im2col_codes(act, B, H, H, Cin, Cin, k, k, stride, pad, cols, ld)
+        R.rmsmp_gemm_workspace(lay, pk, ws, cols, N, ld, 0.1, y, M, R.OUT_NM, None)
+    ms = timed(first_layer)
+    record("resnet-18 conv1 7x7 s2 (3 channels, patch matrix + linear layer) 224x224 B=%d" % B, lay, ms, 2 * M * K * N,
+           (lay.nP + lay.nF4) * K // 2 + lay.n8 * K + 8 * M + B * H * H * Cin + 4 * N * M)
     return rows
 
 

@@ -247,6 +247,26 @@ rmsmp_status rmsmp_conv_depthwise(const rmsmp_layer* layer, const void* d_packed
                                   int32_t* d_acc, void* stream);
 
 /*
+ * Patch matrix of a convolution with few input channels (a network's first layer: 3 channels,
+ * 7 x 7 filters, stride 2; Section 4.1 and Table 6 quantize that layer like all others).  The
+ * implicit form fetches one filter tap per bulk copy, which needs 16 bytes of channels per pixel;
+ * a 3-channel layer is instead run as a linear layer over its patches:
+ *   d_cols[n][(i * kw + j) * C + c] = d_act[b][ho * stride + i - pad][wo * stride + j - pad][c]
+ * for output pixel n = (b * Ho + ho) * Wo + wo, zero outside the image and in the columns from
+ * kh * kw * C up to ld_cols.  The layer's weights are packed as a linear layer with K = ld_cols
+ * in the same order ([M][kh][kw][C], zero columns appended), and rmsmp_gemm* on d_cols with
+ * N = B * Ho * Wo gives the convolution's [N][M] output.
+ *   d_act    device, int8 codes [B][H][W] pixels of pix_pitch bytes, the first C of which are used
+ *   d_cols   device, 16-byte aligned, [B*Ho*Wo][ld_cols]; ld_cols a multiple of 16, >= kh*kw*C
+ * Limits: C <= 64, kh, kw <= 16, stride 1..8, pad 0..16, ld_cols <= 4096.  Allocates nothing; one kernel
+ * on `stream`.
+ * Errors: NULL, SHAPE (limits, ld_cols too small, more than 2^31 pixels), ALIGN, ARCH, CUDA.
+ */
+rmsmp_status rmsmp_im2col_codes(const int8_t* d_act, int B, int H, int W, int C, int64_t pix_pitch,
+                                int kh, int kw, int stride, int pad, int8_t* d_cols, int64_t ld_cols,
+                                void* stream);
+
+/*
  * Many small-batch linear layers in one launch (Algorithm 1's forward line, layer after layer;
  * Section 3.1: the layers execute one after another on the same hardware).  With a
  * handful of tokens a layer is bound by reading its packed weights once, which takes a fraction

@@ -170,6 +170,27 @@ def conv(values, act, stride: int, pad: int) -> np.ndarray:
     return acc
 
 
+def im2col(act, kh: int, kw: int, stride: int, pad: int, ld: int | None = None) -> np.ndarray:
+    """Patch matrix of act[B][H][W][C]: row (b, ho, wo) holds the kh x kw x C codes its output pixel sees, tap
+    by tap with the channel fastest, zero outside the image and in the columns beyond kh*kw*C (up to ld).  A
+    convolution is the matrix product of the filters, flattened in the same order, with these rows (the
+    first layer of the networks of Section 4.1 is run that way)."""
+    act = _c(act, np.int8)
+    B, H, W, Cc = act.shape
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad)
+    K = kh * kw * Cc
+    cols = np.zeros((B, Ho, Wo, ld or K), np.int8)
+    for b in range(B):
+        for ho in range(Ho):
+            for wo in range(Wo):
+                for i in range(kh):
+                    for j in range(kw):
+                        y, x = ho * stride + i - pad, wo * stride + j - pad
+                        if 0 <= y < H and 0 <= x < W:
+                            cols[b, ho, wo, (i * kw + j) * Cc:(i * kw + j + 1) * Cc] = act[b, y, x]
+    return cols.reshape(B * Ho * Wo, -1)
+
+
 def conv_depthwise(values, act, stride: int, pad: int) -> np.ndarray:
     """values[C][kh][kw] int8, act[B][H][W][C] int8 -> acc[B][Ho][Wo][C] int32 (each channel with its own filter)."""
     values, act = _c(values, np.int8), _c(act, np.int8)

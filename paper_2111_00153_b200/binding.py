@@ -32,7 +32,7 @@ EXPORTS = (
     "rmsmp_measure_mma_peak", "rmsmp_workspace_bytes", "rmsmp_expand_weights", "rmsmp_gemm_workspace",
     "rmsmp_conv_implicit_workspace", "rmsmp_gemm_builtin_scratch", "rmsmp_grouped_table_bytes",
     "rmsmp_gemm_grouped", "rmsmp_gemm_workspace_requant", "rmsmp_conv_implicit_workspace_requant",
-    "rmsmp_conv_depthwise", "rmsmp_layer_init_ratio", "rmsmp_assign_scratch_bytes", "rmsmp_assign_quantize_pack", "rmsmp_selftest_bounded_wait", "rmsmp_grouped_plan_bytes", "rmsmp_gemm_grouped_prepare", "rmsmp_gemm_grouped_launch",
+    "rmsmp_conv_depthwise", "rmsmp_im2col_codes", "rmsmp_layer_init_ratio", "rmsmp_assign_scratch_bytes", "rmsmp_assign_quantize_pack", "rmsmp_selftest_bounded_wait", "rmsmp_grouped_plan_bytes", "rmsmp_gemm_grouped_prepare", "rmsmp_gemm_grouped_launch",
 )
 
 
@@ -125,6 +125,7 @@ def lib() -> C.CDLL:
         L.rmsmp_conv_implicit_workspace_requant.argtypes = [C.POINTER(rmsmp_layer), vp, vp, vp, i32, i32, i32, i32, i32,
                                                             f32, f32, i32, vp, C.POINTER(C.c_float), vp]
         L.rmsmp_conv_depthwise.argtypes = [C.POINTER(rmsmp_layer), vp, vp, i32, i32, i32, i32, i32, f32, vp, vp, vp]
+        L.rmsmp_im2col_codes.argtypes = [vp, i32, i32, i32, i32, C.c_int64, i32, i32, i32, i32, vp, C.c_int64, vp]
         L.rmsmp_layer_init_ratio.argtypes = [C.POINTER(rmsmp_layer), i32, i32, i32, i32, i32, i32, i32]
         L.rmsmp_assign_scratch_bytes.argtypes = [i32, C.POINTER(C.c_size_t)]
         L.rmsmp_assign_quantize_pack.argtypes = [vp, i32, C.POINTER(rmsmp_layer), i32, i32, i32, vp, i32, vp, C.c_size_t,
@@ -361,6 +362,12 @@ def rmsmp_conv_depthwise(layer, d_packed, d_act, B: int, H: int, W: int, stride:
                          d_out, d_acc=None, stream=None):
     _check(lib().rmsmp_conv_depthwise(C.byref(layer), _dp(d_packed), _dp(d_act), B, H, W, stride, pad, act_step,
                                       _dp(d_out), _dp(d_acc), _stream(stream)), "rmsmp_conv_depthwise")
+
+
+def rmsmp_im2col_codes(d_act, B: int, H: int, W: int, Cc: int, pix_pitch: int, kh: int, kw: int, stride: int, pad: int,
+                       d_cols, ld_cols: int, stream=None):
+    _check(lib().rmsmp_im2col_codes(_dp(d_act), B, H, W, Cc, pix_pitch, kh, kw, stride, pad, _dp(d_cols), ld_cols,
+                                    _stream(stream)), "rmsmp_im2col_codes")
 
 
 def rmsmp_layer_init_ratio(M: int, Cin: int, kh: int, kw: int, ratio) -> rmsmp_layer:

@@ -8,7 +8,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "librmsmp.so")
-SOURCES = ("host_api.cu", "pack.cu", "simt.cu", "tensor.cu", "tensor2.cu", "peak.cu", "builtin_scratch.cu", "stream.cu", "assign.cu", "depthwise.cu")
+SOURCES = ("host_api.cu", "pack.cu", "simt.cu", "tensor.cu", "tensor2.cu", "peak.cu", "builtin_scratch.cu", "stream.cu", "assign.cu", "depthwise.cu", "gather.cu")
 HEADERS = tuple(sorted(f for f in os.listdir(CSRC) if f.endswith((".cuh", ".h")))) + \
           (os.path.join("..", "..", "include", "rmsmp.h"),)
 
@@ -17,6 +17,7 @@ NVCC_FLAGS = [
     "--fmad=false",                       # quantizer arithmetic is one IEEE operation per step
     "-Xcompiler", "-fPIC,-ffp-contract=off,-O2",
     "-shared",
+    "-ldl",                               # the NVTX header loads a profiler's library on demand
 ]
 
 

@@ -91,6 +91,9 @@ cudaError_t launch_pack(const float* dW, int conv_oihw, const rmsmp_layer& L, in
 // depthwise convolution on the CUDA cores (depthwise.cu)
 bool depthwise_supported(const Problem& p);
 cudaError_t launch_depthwise(const Problem& p, cudaStream_t st);
+// patch matrix of a few-channel convolution (gather.cu)
+cudaError_t launch_im2col(const int8_t* act, int B, int H, int W, int C, int64_t pix_pitch, int kh, int kw, int stride, int pad,
+                          int Ho, int Wo, int8_t* cols, int64_t ld_cols, cudaStream_t st);
 // row assignment on the device + the packed buffer's metadata (assign.cu); scratch of assign_scratch_bytes(M)
 size_t assign_scratch_bytes(int M);
 cudaError_t launch_assign_meta(const float* dW, const rmsmp_layer& L, const float* d_alpha, int pot_mode, uint8_t* blob,

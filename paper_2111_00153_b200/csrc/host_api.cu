@@ -149,6 +149,17 @@ rmsmp_status dispatch(Problem& p, rmsmp_variant variant, cudaStream_t st)
 
 }  // namespace
 
+#include <nvtx3/nvToolsExt.h>
+
+// A named NVTX range around every call that queues GPU work: a profiler's timeline shows which API call a
+// kernel belongs to.  Without a tool attached the two calls return at once.
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange&) = delete;
+    NvtxRange& operator=(const NvtxRange&) = delete;
+};
+
 namespace rmsmp {
 
 int device_ordinal()
@@ -330,6 +341,7 @@ rmsmp_status rmsmp_assign_quantize_pack(const float* d_W, rmsmp_w_layout w_layou
                                         size_t packed_bytes, void* d_scratch, size_t scratch_bytes, uint8_t* d_scheme,
                                         uint8_t* d_bits, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_assign_quantize_pack");
     if (!d_W || !L || !d_packed || !d_scratch) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     if (L->M > 65536 || A < 0 || B < 0 || C < 0 || A + B + C != 100) return RMSMP_ERR_SHAPE;
@@ -357,6 +369,7 @@ rmsmp_status rmsmp_quantize_pack(const float* d_W, rmsmp_w_layout w_layout, cons
                                  const float* h_alpha, rmsmp_pot_mode pot_mode, void* d_packed,
                                  size_t packed_bytes, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_quantize_pack");
     if (!d_W || !L || !h_scheme || !h_bits || !h_alpha || !d_packed) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     if (w_layout != RMSMP_W_LINEAR && w_layout != RMSMP_W_CONV_OIHW) return RMSMP_ERR_SHAPE;
@@ -422,6 +435,7 @@ rmsmp_status rmsmp_quantize_pack(const float* d_W, rmsmp_w_layout w_layout, cons
 rmsmp_status rmsmp_unpack_codes(const rmsmp_layer* L, const void* d_packed, int8_t* d_values,
                                 int32_t* d_perm, float* d_wstep, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_unpack_codes");
     if (!L || !d_packed || !d_values) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     rmsmp_status a = check_arch();
@@ -437,6 +451,7 @@ rmsmp_status rmsmp_unpack_codes(const rmsmp_layer* L, const void* d_packed, int8
 rmsmp_status rmsmp_quantize_act(const float* d_X, size_t count, float alpha_a, rmsmp_act_kind kind,
                                 int8_t* d_codes, float* h_act_step, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_quantize_act");
     if (!d_X || !d_codes) return RMSMP_ERR_NULL;
     if (count < 1) return RMSMP_ERR_SHAPE;
     if (kind != RMSMP_ACT_U4 && kind != RMSMP_ACT_S4) return RMSMP_ERR_SCHEME;
@@ -558,6 +573,7 @@ static rmsmp_status grouped_problems(const rmsmp_gemm_item* h_items, int count, 
 rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
                                 void* d_table, size_t table_bytes, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_gemm_grouped");
     if (!d_table) return RMSMP_ERR_NULL;
     std::vector<Problem> probs;
     rmsmp_status s = grouped_problems(h_items, count, out_layout, probs);
@@ -617,6 +633,7 @@ rmsmp_status rmsmp_grouped_plan_bytes(const rmsmp_gemm_item* h_items, int count,
 rmsmp_status rmsmp_gemm_grouped_prepare(const rmsmp_gemm_item* h_items, int count, rmsmp_out_layout out_layout,
                                         void* d_table, size_t table_bytes, rmsmp_grouped_plan* plan, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_gemm_grouped_prepare");
     if (!d_table || !plan) return RMSMP_ERR_NULL;
     std::memset(plan, 0, sizeof(*plan));
     std::vector<Problem> probs;
@@ -653,6 +670,7 @@ rmsmp_status rmsmp_gemm_grouped_prepare(const rmsmp_gemm_item* h_items, int coun
 
 rmsmp_status rmsmp_gemm_grouped_launch(const rmsmp_grouped_plan* plan, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_gemm_grouped_launch");
     if (!plan) return RMSMP_ERR_NULL;
     if (plan->magic != kPlanMagicHost || !plan->d_table || plan->grid < 1) return RMSMP_ERR_BAD_LAYER;
     rmsmp_status a = check_arch();
@@ -672,6 +690,7 @@ rmsmp_status rmsmp_gemm_variant(const rmsmp_layer* L, const void* d_packed, cons
                                 int64_t ld_out, rmsmp_out_layout out_layout, int32_t* d_acc,
                                 rmsmp_variant variant, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_gemm_variant");
     return gemm_impl(L, d_packed, nullptr, false, d_act, N, ld_act, act_step, d_out, ld_out, out_layout, d_acc,
                      variant, stream);
 }
@@ -681,6 +700,7 @@ rmsmp_status rmsmp_gemm_workspace(const rmsmp_layer* L, const void* d_packed, co
                                   float* d_out, int64_t ld_out, rmsmp_out_layout out_layout,
                                   int32_t* d_acc, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_gemm_workspace");
     return gemm_impl(L, d_packed, d_workspace, true, d_act, N, ld_act, act_step, d_out, ld_out, out_layout,
                      d_acc, RMSMP_VARIANT_TENSOR, stream);
 }
@@ -689,6 +709,7 @@ rmsmp_status rmsmp_gemm(const rmsmp_layer* L, const void* d_packed, const int8_t
                         int64_t ld_act, float act_step, float* d_out, int64_t ld_out,
                         rmsmp_out_layout out_layout, int32_t* d_acc, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_gemm");
     return rmsmp_gemm_variant(L, d_packed, d_act, N, ld_act, act_step, d_out, ld_out, out_layout,
                               d_acc, RMSMP_VARIANT_AUTO, stream);
 }
@@ -731,6 +752,7 @@ static rmsmp_status conv_impl(const rmsmp_layer* L, const void* d_packed, const 
 rmsmp_status rmsmp_conv_depthwise(const rmsmp_layer* L, const void* d_packed, const int8_t* d_act, int B, int H, int W,
                                   int stride, int pad, float act_step, float* d_out, int32_t* d_acc, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_conv_depthwise");
     if (!L || !d_packed || !d_act || !d_out) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     if (L->Cin != 1) return RMSMP_ERR_SHAPE;              // a depthwise layer is described as M = channels, Cin = 1
@@ -758,12 +780,35 @@ rmsmp_status rmsmp_conv_depthwise(const rmsmp_layer* L, const void* d_packed, co
     return RMSMP_OK;
 }
 
+rmsmp_status rmsmp_im2col_codes(const int8_t* d_act, int B, int H, int W, int C, int64_t pix_pitch, int kh, int kw,
+                                int stride, int pad, int8_t* d_cols, int64_t ld_cols, void* stream)
+{
+    NvtxRange nvtx_range("rmsmp_im2col_codes");
+    if (!d_act || !d_cols) return RMSMP_ERR_NULL;
+    if (B < 1 || H < 1 || W < 1 || C < 1 || C > 64 || kh < 1 || kw < 1 || kh > 16 || kw > 16) return RMSMP_ERR_SHAPE;
+    if (stride < 1 || stride > 8 || pad < 0 || pad > 16 || pix_pitch < C) return RMSMP_ERR_SHAPE;
+    if (H + 2 * pad < kh || W + 2 * pad < kw) return RMSMP_ERR_SHAPE;
+    if (ld_cols < (int64_t)kh * kw * C || ld_cols > 4096) return RMSMP_ERR_SHAPE;
+    const int Ho = (H + 2 * pad - kh) / stride + 1, Wo = (W + 2 * pad - kw) / stride + 1;
+    if ((int64_t)B * Ho * Wo > (int64_t)1 << 31 || (int64_t)B * H * W > (int64_t)1 << 31) return RMSMP_ERR_SHAPE;
+    if (!aligned16(d_cols) || (ld_cols & 15)) return RMSMP_ERR_ALIGN;
+    rmsmp_status a = check_arch();
+    if (a != RMSMP_OK) return a;
+    if (launch_im2col(d_act, B, H, W, C, pix_pitch, kh, kw, stride, pad, Ho, Wo, d_cols, ld_cols,
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return RMSMP_ERR_CUDA;
+    }
+    return RMSMP_OK;
+}
+
 rmsmp_status rmsmp_conv_implicit_variant(const rmsmp_layer* L, const void* d_packed,
                                          const int8_t* d_act, int B, int H, int W, int stride,
                                          int pad, float act_step, float* d_out,
                                          rmsmp_out_layout out_layout, int32_t* d_acc,
                                          rmsmp_variant variant, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_conv_implicit_variant");
     return conv_impl(L, d_packed, nullptr, false, d_act, B, H, W, stride, pad, act_step, d_out, out_layout,
                      d_acc, variant, stream);
 }
@@ -773,6 +818,7 @@ rmsmp_status rmsmp_conv_implicit_workspace(const rmsmp_layer* L, const void* d_p
                                            int W, int stride, int pad, float act_step, float* d_out,
                                            rmsmp_out_layout out_layout, int32_t* d_acc, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_conv_implicit_workspace");
     return conv_impl(L, d_packed, d_workspace, true, d_act, B, H, W, stride, pad, act_step, d_out, out_layout,
                      d_acc, RMSMP_VARIANT_TENSOR, stream);
 }
@@ -782,6 +828,7 @@ rmsmp_status rmsmp_gemm_workspace_requant(const rmsmp_layer* L, const void* d_pa
                                           float next_alpha, rmsmp_act_kind next_kind, int8_t* d_next_codes,
                                           int64_t ld_codes, float* h_next_step, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_gemm_workspace_requant");
     const Requant rq = {next_alpha, next_kind, d_next_codes, ld_codes};
     rmsmp_status s = requant_check(&rq, h_next_step);
     if (s != RMSMP_OK) return s;
@@ -795,6 +842,7 @@ rmsmp_status rmsmp_conv_implicit_workspace_requant(const rmsmp_layer* L, const v
                                                    rmsmp_act_kind next_kind, int8_t* d_next_codes,
                                                    float* h_next_step, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_conv_implicit_workspace_requant");
     const Requant rq = {next_alpha, next_kind, d_next_codes, 0};
     rmsmp_status s = requant_check(&rq, h_next_step);
     if (s != RMSMP_OK) return s;
@@ -813,6 +861,7 @@ rmsmp_status rmsmp_workspace_bytes(const rmsmp_layer* L, size_t* bytes)
 rmsmp_status rmsmp_expand_weights(const rmsmp_layer* L, const void* d_packed, void* d_workspace,
                                   size_t workspace_bytes, void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_expand_weights");
     if (!L || !d_packed || !d_workspace) return RMSMP_ERR_NULL;
     if (!layer_ok(L)) return RMSMP_ERR_BAD_LAYER;
     if (workspace_bytes < (size_t)L->M * L->Kp) return RMSMP_ERR_BUFFER_TOO_SMALL;
@@ -832,6 +881,7 @@ rmsmp_status rmsmp_conv_implicit(const rmsmp_layer* L, const void* d_packed, con
                                  float* d_out, rmsmp_out_layout out_layout, int32_t* d_acc,
                                  void* stream)
 {
+    NvtxRange nvtx_range("rmsmp_conv_implicit");
     return rmsmp_conv_implicit_variant(L, d_packed, d_act, B, H, W, stride, pad, act_step, d_out,
                                        out_layout, d_acc, RMSMP_VARIANT_AUTO, stream);
 }

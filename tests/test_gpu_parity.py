@@ -623,3 +623,58 @@ def test_depthwise_conv_rejects_what_it_cannot_run():
     with pytest.raises(R.RmsmpError) as e:
         R.rmsmp_conv_depthwise(layer, d_packed, a, 1, 4, 4, 1, 1, 0.1, y)
     assert e.value.status == R.ERR_SHAPE
+
+
+# ---------------------------------------------------------------- first layer (few channels) as a patch matrix
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,Cin,k,stride,pad,B,H,W,pitch", [
+    (64, 3, 7, 2, 3, 2, 30, 26, 3),        # the networks' first layer (Section 4.1): 3 channels, 7 x 7, stride 2
+    (24, 3, 3, 1, 1, 1, 9, 7, 4),          # a padded pixel pitch
+    (40, 1, 5, 1, 0, 2, 8, 8, 1),
+    (16, 64, 3, 1, 1, 1, 4, 262, 64),      # input rows too wide for shared memory: the direct-gather form
+])
+def test_first_layer_patch_matrix_and_gemm_match_oracle_conv(M, Cin, k, stride, pad, B, H, W, pitch):
+    import torch
+    g = synth.rng(91, M + Cin + H)
+    Wt = synth.weights_normal(g, (M, Cin, k, k))
+    scheme, bits = O.assign_rows(Wt.reshape(M, -1), (60, 35, 5))
+    alpha = synth.alpha_rows(Wt.reshape(M, -1))
+    act = synth.act_codes_uniform(g, (B, H, W, Cin))
+    K = k * k * Cin
+    ld = (K + 15) // 16 * 16
+    # patch matrix on the device against the oracle's
+    a = torch.zeros((B, H, W, pitch), dtype=torch.int8, device="cuda")
+    a[..., :Cin] = torch.from_numpy(act).cuda()
+    Ho, Wo = O.conv_out_hw(H, W, k, k, stride, pad)
+    N = B * Ho * Wo
+    cols = torch.full((N, ld), 99, dtype=torch.int8, device="cuda")
+    R.rmsmp_im2col_codes(a, B, H, W, Cin, pitch, k, k, stride, pad, cols, ld)
+    torch.cuda.synchronize()
+    assert np.array_equal(cols.cpu().numpy(), O.im2col(act, k, k, stride, pad, ld))
+    # the layer as a linear layer over the patches, filters flattened tap-major with zero columns appended
+    Wl = np.zeros((M, ld), np.float32)
+    Wl[:, :K] = Wt.transpose(0, 2, 3, 1).reshape(M, K)
+    layer, d_packed = Hn.pack_layer(Wl, scheme, bits, alpha)
+    step = np.float32(0.05)
+    y = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+    acc = torch.zeros((N, M), dtype=torch.int32, device="cuda")
+    R.rmsmp_gemm_variant(layer, d_packed, cols, N, ld, float(step), y, M, R.OUT_NM, acc, R.VARIANT_AUTO)
+    torch.cuda.synchronize()
+    assert R.rmsmp_last_device_status(d_packed) == R.OK
+    _, _, acc_ref, y_ref = O.layer_conv(Wt, scheme, bits, alpha, act, step, stride, pad)
+    assert np.array_equal(acc.cpu().numpy(), acc_ref.reshape(N, M))
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.reshape(N, M).view(np.uint32))
+
+
+@pytest.mark.gpu
+def test_patch_matrix_rejects_bad_arguments():
+    import torch
+    a = torch.zeros((1, 4, 4, 3), dtype=torch.int8, device="cuda")
+    cols = torch.zeros((16, 32), dtype=torch.int8, device="cuda")
+    for args, status in [((a, 1, 4, 4, 3, 3, 3, 3, 1, 1, cols, 16), R.ERR_SHAPE),       # ld_cols below kh*kw*C
+                         ((a, 1, 4, 4, 3, 3, 3, 3, 1, 1, cols, 40), R.ERR_ALIGN),       # not a multiple of 16
+                         ((a, 1, 4, 4, 3, 2, 3, 3, 1, 1, cols, 32), R.ERR_SHAPE),       # pitch below the channel count
+                         ((a, 1, 4, 4, 3, 3, 7, 7, 1, 0, cols, 160), R.ERR_SHAPE)]:     # filter larger than the image
+        with pytest.raises(R.RmsmpError) as e:
+            R.rmsmp_im2col_codes(*args)
+        assert e.value.status == status

@@ -432,3 +432,20 @@ def test_depthwise_conv_is_the_dense_conv_with_block_diagonal_filters():
                 if 0 <= y < H and 0 <= x < W:
                     s += int(v[c, i, j]) * int(a[b, y, x, c])
         assert got[b, ho, wo, c] == s
+
+
+def test_patch_matrix_times_flattened_filters_is_the_convolution():
+    """im2col against the direct convolution (a different code path: the C loop nest), over stride, padding and
+    an odd channel count; and its zero padding and column order on a hand-made case."""
+    g = np.random.default_rng(41)
+    for (Cin, k, stride, pad, H, W) in [(3, 7, 2, 3, 11, 9), (3, 3, 1, 1, 5, 6), (5, 2, 2, 0, 6, 6), (1, 3, 1, 2, 4, 4)]:
+        V = g.integers(-7, 8, (6, Cin, k, k), dtype=np.int8)
+        act = g.integers(-8, 16, (2, H, W, Cin), dtype=np.int8)
+        cols = O.im2col(act, k, k, stride, pad, ld=(k * k * Cin + 15) // 16 * 16)
+        Vl = np.zeros((6, cols.shape[1]), np.int8)
+        Vl[:, :k * k * Cin] = V.transpose(0, 2, 3, 1).reshape(6, -1)
+        assert np.array_equal(O.matmul(Vl, cols), O.conv(V, act, stride, pad).reshape(-1, 6))
+        assert not cols[:, k * k * Cin:].any()
+    # one pixel, 2 channels (codes 5, 6), 2 x 2 filter, pad 1: four output pixels, each seeing the pixel at another tap
+    cols = O.im2col(np.array([[[[5, 6]]]], np.int8), 2, 2, 1, 1)
+    assert cols.tolist() == [[0, 0, 0, 0, 0, 0, 5, 6], [0, 0, 0, 0, 5, 6, 0, 0], [0, 0, 5, 6, 0, 0, 0, 0], [5, 6, 0, 0, 0, 0, 0, 0]]
