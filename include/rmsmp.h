@@ -57,7 +57,9 @@ typedef enum { RMSMP_W_LINEAR = 0, RMSMP_W_CONV_OIHW = 1 } rmsmp_w_layout;
 /* Which kernel carries out the contraction. */
 typedef enum {
     RMSMP_VARIANT_AUTO = 0,      /* library picks by shape */
-    RMSMP_VARIANT_TENSOR = 1,    /* TMA + in-smem code expansion + tcgen05 int8 MMA, TMEM accumulators */
+    RMSMP_VARIANT_TENSOR = 1,    /* TMA + in-smem code expansion + tcgen05 int8 MMA, TMEM accumulators.  A layer of one
+                                    128-row block whose expanded weights fit 72 KB is expanded ONCE per CTA into
+                                    resident shared memory; longer rows are expanded k-block by k-block per tile */
     RMSMP_VARIANT_SIMT = 2,      /* CUDA-core integer multiply-add (dp4a) on codes expanded in registers */
     RMSMP_VARIANT_SHIFTADD = 3,  /* CUDA cores; PoT rows by shift-and-add, no multiplier */
     RMSMP_VARIANT_SIMPLE = 4     /* one thread per output, scalar; bring-up / cross-check */

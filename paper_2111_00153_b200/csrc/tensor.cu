@@ -72,6 +72,8 @@ struct TensorCfg {
     int bk;                // codes per k-block and bytes per operand row in shared memory: 128, or 64 (pre mode,
                            //    channel counts that would leave half of a 128-byte row empty)
     int a_bytes, b_bytes;  // one A / B stage
+    int fill;              // 1 (resident weights, no workspace given): the CTA expands its row block from the packed codes
+                           //    itself, once, instead of copying expanded weights in
     int ares;              // 1 (pre mode, one row block, small K): the expanded weights of all k-blocks are loaded once
                            //    per CTA and stay in shared memory; only activation boxes flow through a ring
     int m2;                // 1 (pre mode, even number of row blocks): a tile covers TWO row blocks.  Both use the same
@@ -156,6 +158,65 @@ __device__ __forceinline__ void expand_task(uint32_t meta, uint32_t raw_stage, u
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst ^ 16u), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
 
+// Resident weights without a workspace: every thread of the CTA expands 16-code granules of the row block
+// from the packed codes (exact int8 values, as expand_kernel writes them) straight into the resident stages,
+// at the place the bulk copy of an expanded [rows][bk] box would have put them: stage kb = (tap, channel
+// chunk) holds codes [tap * Cp + chunk * bk, + bk) of every row, 16-byte units XOR-swizzled by the row
+// (128-byte rows: unit ^ (row & 7); 64-byte rows: unit ^ ((row >> 1) & 3)), zeros beyond M and Kp; with
+// duplicated rows (M <= 64) a second copy goes to lanes 64..127.
+__device__ __forceinline__ void fill_resident_weights(const Problem& p, const TensorCfg& cfg, uint32_t sA, int tid, int nthreads)
+{
+    const int rows = cfg.dup ? kBlockRows / 2 : kBlockRows;
+    const int gpr = cfg.bk >> 4;
+    const int n4 = p.nP + p.nF4;
+    // a few threads per row, each with every tpr-th granule of it: kind and place of the row are read once, and a
+    // thread's loads are independent of one another
+    const int tpr = nthreads / rows;
+    const int r = tid / tpr, sub = tid - r * tpr;
+    if (r < rows) {
+        const bool have = r < p.M;
+        const int kind = have ? (int)p.kind[r] : kFixed8;
+        const int slot = have ? p.slot[r] : 0;
+        const uint8_t* src = (kind == kFixed8) ? p.q8 + (size_t)(have ? slot - n4 : 0) * p.Kp : p.q4 + (size_t)slot * (p.Kp >> 1);
+        const uint32_t phase = (cfg.bk == 128) ? (uint32_t)(r & 7) : (uint32_t)((r >> 1) & 3);
+        const uint32_t row_base = sA + (uint32_t)r * (uint32_t)cfg.bk;
+        const int gtot = cfg.nkb * gpr;
+#pragma unroll 4
+        for (int g = sub; g < gtot; g += tpr) {
+            const int kb = g / gpr, q = g - kb * gpr;
+            const int tap = kb / cfg.cpt, cc = kb - tap * cfg.cpt;
+            const int k = tap * p.Cp + cc * cfg.bk + q * 16;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (have && k < p.Kp) {
+                if (kind == kFixed8) {
+                    v = __ldg(reinterpret_cast<const uint4*>(src + k));
+                } else {
+                    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(src + ((k >> 5) << 4)));
+                    uint32_t w[8];
+                    if (kind == kPoT4) {
+                        expand_pot_chunk(raw, w);
+                    } else {
+                        expand_fixed4_chunk_x16(raw, w);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {       // 16 * value -> value: shift every byte right by four, keeping its sign
+                            const uint32_t x = w[j];
+                            w[j] = ((x >> 4) & 0x0F0F0F0Fu) | (((x >> 7) & 0x01010101u) * 0xF0u);
+                        }
+                    }
+                    const int h = (k >> 4) & 1;
+                    v = h ? make_uint4(w[4], w[5], w[6], w[7]) : make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            const uint32_t dst = row_base + (uint32_t)kb * (uint32_t)cfg.a_bytes + (((uint32_t)q ^ phase) << 4);
+            // (no memory clobber: the loads of the next granules may move above these stores)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
+            if (cfg.dup)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)(cfg.a_bytes / 2)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the MMAs read these bytes through the async proxy
+}
+
 // ------------------------------------------------------------------ the kernel
 
 // kM2: a tile covers two row blocks (TensorCfg::m2), compiled separately so that the common form keeps its registers.
@@ -220,13 +281,21 @@ tensor_kernel(const Problem p, const TensorCfg cfg, const __grid_constant__ Maps
     const int64_t first = blockIdx.x, step = gridDim.x;
     const int64_t my_tiles = (cfg.ntiles > first) ? (cfg.ntiles - first + step - 1) / step : 0;
 
+    if (kAres && cfg.fill && warp != 0) {
+        // every warp but the activation producer's (whose first copies go out meanwhile) expands the row block;
+        // one of them then reports the resident weights to the MMA thread
+        if (my_tiles > 0) fill_resident_weights(p, cfg, sA, (int)threadIdx.x - 32, kThreads - 32);
+        asm volatile("bar.sync 1, %0;" ::"n"(kThreads - 32) : "memory");
+        if (threadIdx.x == 32 && my_tiles > 0) mbar_arrive(bar_fullA);
+    }
+
     // Workspace mode splits the producer: one thread can start a bulk tensor copy only every few
     // hundred cycles, so the activation boxes and the weight boxes are issued by two different warps.
     const bool pre_b_producer = kPre && warp == 0;
     const bool pre_a_producer = kPre && !kAres && warp == 2;
     if (pre_b_producer || pre_a_producer) {
         if (lane == 0) {
-            if (pre_b_producer && kAres && my_tiles > 0) {
+            if (pre_b_producer && kAres && my_tiles > 0 && !cfg.fill) {
                 // resident weights: every k-block's rows, once
                 mbar_arrive_expect_tx(bar_fullA, (uint32_t)(cfg.nkb * cfg.a_bytes));
                 int tap = 0, cc = 0;
@@ -842,6 +911,14 @@ bool plan(const Problem& p, TensorCfg& c)
     c.b_sub = 0;
     c.colshift = 0;
     c.pre = p.wexp ? 1 : 0;
+    c.fill = 0;
+    if (!p.wexp && p.nblocks == 1 && !p.rq_codes) {
+        // no workspace, but the whole row block's expanded weights would stay resident: the CTA expands them once
+        // itself and the layer runs in the workspace form
+        const int bk = ((p.Cin % 128 != 0) && (p.Cin % 128 <= 64)) ? 64 : 128;
+        const int64_t nkb = (int64_t)p.kh * p.kw * ((p.Cin + bk - 1) / bk);
+        if (nkb * kBlockRows * bk <= 72 * 1024) { c.pre = 1; c.fill = 1; }
+    }
     // 64-byte k-blocks when a 128-byte row would be at most half used by the (last) channel chunk
     c.bk = (c.pre && (p.Cin % 128 != 0) && (p.Cin % 128 <= 64)) ? 64 : 128;
     c.a_bytes = kBlockRows * c.bk;
