@@ -343,6 +343,41 @@ def test_grouped_tensor_launch_rejects_what_it_cannot_run():
     with pytest.raises(R.RmsmpError) as e:
         R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table[:256])
     assert e.value.status == R.ERR_BUFFER_TOO_SMALL
+    # PoT rows are summed in fp32 on the tensor core: exact up to a reduction length of 16384, refused beyond
+    keep, items, refs = _grouped_case([(16, 16384 + 128)], 2)
+    arr = R.make_gemm_items(items)
+    table2 = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
+    with pytest.raises(R.RmsmpError) as e:
+        R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table2)
+    assert e.value.status == R.ERR_VARIANT
+
+
+def test_grouped_tensor_launch_longest_exact_reduction_with_extreme_codes():
+    """K = 16384, every weight at full scale (PoT rows: +-64 in units of the row's step), every activation 15 or
+    -16: the fp32 sums of the PoT tiles reach their largest magnitude (2^24 - 2^14 quarter units) and must still
+    be the exact integers."""
+    import torch
+    M, K, N = 40, 16384, 3
+    W = np.ones((M, K), np.float32)
+    W[::3] = -1
+    scheme, bits = O.assign_rows(synth.weights_normal(synth.rng(5, 77), (M, K)), (60, 35, 5))
+    alpha = np.ones(M, np.float32)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    v_ref, wstep = O.quantize_rows(W, scheme, bits, alpha)
+    for codes, nonneg in ((np.full((N, K), 15, np.int8), 1), (np.full((N, K), -16, np.int8), 0), (np.full((N, K), 15, np.int8), 0)):
+        a = torch.from_numpy(codes).cuda()
+        y = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+        acc = torch.zeros((N, M), dtype=torch.int32, device="cuda")
+        arr = R.make_gemm_items([(layer, d_packed, a, N, K, 1.0, y, M, acc, nonneg)])
+        table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
+        plan = R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table)
+        R.rmsmp_gemm_grouped_launch(plan)
+        torch.cuda.synchronize()
+        assert R.rmsmp_last_device_status(d_packed) == R.OK
+        acc_ref = O.matmul(v_ref, codes)
+        assert np.abs(acc_ref).max() >= 64 * 15 * K
+        assert np.array_equal(acc.cpu().numpy(), acc_ref)
+        assert np.array_equal(y.cpu().numpy().view(np.uint32), _expected(acc_ref, wstep, np.float32(1.0)).view(np.uint32))
     with pytest.raises(R.RmsmpError) as e:
         R.rmsmp_gemm_grouped_launch(R.rmsmp_grouped_plan())
     assert e.value.status == R.ERR_BAD_LAYER
