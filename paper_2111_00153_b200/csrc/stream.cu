@@ -702,6 +702,10 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
     // accumulator buffers the issuers do not wait for it
     H->nAcc = H->acc_cols <= 64 ? 4 : 2;
     H->nAst = std::min(6, (512 - H->nAcc * H->acc_cols) / kAStageCols) & ~1;      // even: the two expander sets alternate
+    // An issuer waits on the barriers of its own stages only and tells their phases apart by parity, so it must never
+    // skip two phases of a barrier: not more issuers than A stages, and an even number of A stages (each expander set
+    // and each issuer then keeps to its own ones).
+    if (H->nAst < H->nch || H->nAst < 2) return false;
     H->b_bytes = (uint32_t)(2 * H->n_pad * 128);
     H->stage_bytes = 128u * 128u;                                 // one box: at most 128 rows x 128 bytes
     // Shared memory: a packed-code slot is held from the moment its copy is started until the expanders have the
