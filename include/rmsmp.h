@@ -330,7 +330,14 @@ rmsmp_status rmsmp_gemm_grouped(const rmsmp_gemm_item* h_items, int count, rmsmp
  *                               long as the buffers, shapes and leading dimensions the plan was
  *                               built from stay the same (their CONTENTS may change: new weights
  *                               packed with the same row map, new activation codes).  The table
- *                               must stay untouched while launches that use it are in flight.
+ *                               must stay untouched while launches that use it are in flight.  The
+ *                               kernels are launched with the programmatic-stream-serialization
+ *                               attribute and signal early, so that launches in a row overlap their
+ *                               ends and beginnings; what a predecessor may still touch is accessed only
+ *                               behind a grid-dependency wait.  Kernels that follow on the stream and
+ *                               are launched the ordinary way are ordered as always; one that is itself
+ *                               launched with that attribute must call cudaGridDependencySynchronize()
+ *                               before it reads the results.
  * Errors: as rmsmp_gemm_grouped; BAD_LAYER for a plan that was not prepared, or was prepared on
  * another device.
  */

@@ -434,3 +434,31 @@ def test_cta_pair_conv_full(M, Cin, k, stride, pad, B, H):
     codes, step, y = _run_conv_device(W, scheme, bits, alpha, x, stride, pad, R.ACT_U4)
     _, ws, acc, y_ref = O.layer_conv(W, scheme, bits, alpha, codes, step, stride, pad)
     assert np.array_equal(y.view(np.uint32), y_ref.reshape(-1, M).view(np.uint32))
+
+
+def test_grouped_tensor_launches_in_a_row_see_the_inputs_of_their_turn():
+    """Launches of one plan run as programmatic dependents of whatever is in front of them on the stream.  Eight
+    launches in a row, the activation buffers rewritten between them by ordinary kernels and the outputs copied
+    away after each: every launch must have read the codes of its own turn (signed layers through the copy
+    that its first kernel writes) and no launch may have overwritten the outputs of the one before it early."""
+    import torch
+    shapes = [(384, 512), (200, 256), (128, 1024), (130, 96)]
+    N, turns = 5, 8
+    keep, items, refs = _grouped_case(shapes, N)
+    arr = R.make_gemm_items(items)
+    table = torch.empty(R.rmsmp_grouped_plan_bytes(arr), dtype=torch.uint8, device="cuda")
+    plan = R.rmsmp_gemm_grouped_prepare(arr, R.OUT_NM, table)
+    base = [a.clone() for (_, _, a, _, _) in keep]
+    outs = []
+    for t in range(turns):
+        for (layer, d_packed, a, y, acc), b in zip(keep, base):
+            a.copy_(torch.roll(b, t, dims=0))                 # turn t: the tokens rotated by t
+        R.rmsmp_gemm_grouped_launch(plan)
+        if t % 2:
+            R.rmsmp_gemm_grouped_launch(plan)                 # and a launch directly behind a launch
+        outs.append([y.clone() for (_, _, _, y, _) in keep])
+    torch.cuda.synchronize()
+    for t in range(turns):
+        for k, ((acc_ref, y_ref), y) in enumerate(zip(refs, outs[t])):
+            want = np.roll(y_ref, t, axis=0)
+            assert np.array_equal(y.cpu().numpy().view(np.uint32), want.view(np.uint32)), (t, k)
