@@ -708,8 +708,8 @@ def write_traffic_note(csv_path):
     with open(TRAFFIC_NOTE, "w") as f:
         f.write("# DRAM traffic of the %d convolution launches of one step (ResNet-18 stack, batch 256), from the profiler's\n" % n_layers)
         f.write("# launch list: ncu --metrics gpu__time_duration.sum,dram__bytes_read.sum,dram__bytes_write.sum --clock-control none\n")
-        f.write("#   -s 200 -c 200 --csv --log-file gpurun_out/launches.csv python bench.py --steps 2 --warmup 3 --no-e2e --no-cpu-baseline --no-weights-leg\n")
-        f.write("# then: python bench.py --write-traffic-note gpurun_out/launches.csv\n")
+        f.write("#   -s 200 -c 200 --csv --log-file %s python bench.py --steps 2 --warmup 3 --no-e2e --no-cpu-baseline --no-weights-leg\n" % csv_path)
+        f.write("# then: python bench.py --write-traffic-note %s\n" % csv_path)
         f.write("kernel_sources_sha256: %s\n" % kernel_sources_digest())
         f.write("dram_bytes_per_step: %.0f\n" % total)
         f.write("conv_launches: %d\n" % len(step))

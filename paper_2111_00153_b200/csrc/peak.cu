@@ -1,6 +1,6 @@
 // Tensor-pipe ceiling of this GPU for the MMA shape the contraction kernel uses: every SM issues
 // tcgen05.mma (M=128, N=256) back to back on operands that stay in shared memory -- no loads, no
-// epilogue.  kind::i8 (K=32 per instruction) gives the INT8 roofline the layer kernels are judged
+// epilogue.  kind::i8 (K=32 per instruction) gives the INT8 roofline the layer kernels are measured
 // against; kind::f16 with bf16 operands (K=16) calibrates it against the known bf16 figure.
 #include <cuda.h>
 #include "common.cuh"
