@@ -981,6 +981,8 @@ def main():
                          "(config1 .. config5, or 'grouped' for the one-launch BERT-large stack)")
     ap.add_argument("--weights-leg-only", default=None, metavar="TOKENS",
                     help="run only the weight-bound leg at this token count and print it (short: for profiler captures)")
+    ap.add_argument("--second-workloads-only", action="store_true",
+                    help="run only the depthwise / pointwise / bottleneck / first-layer shapes and print their rows (short: for profiler captures)")
     ap.add_argument("--write-traffic-note", default=None, metavar="CSV",
                     help="no GPU work: turn a profiler launch list into the DRAM-traffic note roofline.traffic is read from")
     ap.add_argument("--check-ranks", action="store_true",
@@ -1001,6 +1003,13 @@ def main():
         torch.cuda.set_device(0)
         peaks, _ = load_peaks()
         print(json.dumps(weights_leg(R, torch, peaks, tokens=(int(args.weights_leg_only),), reps=2, launches=3, warm=3)))
+    elif args.second_workloads_only:
+        import torch
+        from paper_2111_00153_b200 import binding as R
+        torch.cuda.set_device(0)
+        peaks, _ = load_peaks()
+        i8, _ = R.rmsmp_measure_mma_peak(torch.zeros(4, dtype=torch.int32, device="cuda"), False, 256, 20000)
+        print(json.dumps(second_workloads_leg(R, torch, peaks, i8)))
     elif args.check_ranks:
         run_check_ranks(args)
     elif args.suite:

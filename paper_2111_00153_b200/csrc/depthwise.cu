@@ -74,21 +74,25 @@ __global__ void __launch_bounds__(kDwThreads, 4) depthwise_kernel(const Problem 
                 int acc[kDwRun][4];
 #pragma unroll
                 for (int r = 0; r < kDwRun; ++r) acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0;
+                // all loads of the run first (rows and columns outside the image read as zero), then the arithmetic
+                uint32_t a[3][kXW];
 #pragma unroll
                 for (int i = 0; i < 3; ++i) {
                     const int y = ho * kS + i - p.pad;
-                    if (y < 0 || y >= p.H) continue;
-                    const int8_t* rowp = img + (size_t)y * p.W * p.pix_pitch;
-                    uint32_t a[kXW];
+                    const bool yin = y >= 0 && y < p.H;
+                    const int8_t* rowp = img + (size_t)(yin ? y : 0) * p.W * p.pix_pitch;
 #pragma unroll
                     for (int xx = 0; xx < kXW; ++xx) {
                         const int x = wo0 * kS + xx - p.pad;
-                        a[xx] = (x >= 0 && x < p.W) ? __ldg(reinterpret_cast<const uint32_t*>(rowp + (size_t)x * p.pix_pitch) + q) : 0u;
+                        a[i][xx] = (yin && x >= 0 && x < p.W) ? __ldg(reinterpret_cast<const uint32_t*>(rowp + (size_t)x * p.pix_pitch) + q) : 0u;
                     }
+                }
+#pragma unroll
+                for (int i = 0; i < 3; ++i) {
 #pragma unroll
                     for (int xx = 0; xx < kXW; ++xx) {
-                        const int a0 = (int)(a[xx] & 0x000000FFu), a1 = (int)(a[xx] & 0x0000FF00u);
-                        const int a2 = (int)(a[xx] & 0x00FF0000u), a3 = (int)(a[xx] & 0xFF000000u);
+                        const int a0 = (int)(a[i][xx] & 0x000000FFu), a1 = (int)(a[i][xx] & 0x0000FF00u);
+                        const int a2 = (int)(a[i][xx] & 0x00FF0000u), a3 = (int)(a[i][xx] & 0xFF000000u);
 #pragma unroll
                         for (int j = 0; j < 3; ++j) {
                             if ((xx - j) % kS != 0 || xx - j < 0 || (xx - j) / kS >= kDwRun) continue;
