@@ -920,7 +920,7 @@ def run_suite(args):
     if want("grouped"):
         leg = weights_leg(R, torch, peaks)
         for r in leg["rows"]:
-            rec = {"suite": "config5", "shape": "bert-large stack, 144 linears, N=%d, one grouped launch (plan prepared once)" % r["tokens"],
+            rec = {"suite": "config5", "shape": "bert-large stack, 144 linears, N=%d, %s codes, one grouped launch (plan prepared once)" % (r["tokens"], r["codes"].split(" ")[0]),
                    "N": r["tokens"], "ratio": list(RATIO), "variant": "grouped_tensor", "us": r["us"], "tops": r["tops"], "gbs": r["gbs"],
                    "frac_int8_peak": r["tops"] / i8_peak, "frac_hbm": r["frac"], "weights": "cold stream"}
             rows.append(rec)
