@@ -288,6 +288,7 @@ stream_kernel(const uint8_t* __restrict__ table)
     const int n_pad = H->n_pad, nS = H->nS, nch = H->nch, nB = H->nB, nAst = H->nAst;
     const uint32_t stage_bytes = H->stage_bytes, b_bytes = H->b_bytes, idesc = H->idesc, idesc_fp = H->idesc_fp;
     const uint32_t acc_cols = (uint32_t)H->acc_cols, nAcc = (uint32_t)H->nAcc, a_base_col = nAcc * acc_cols;
+    const uint32_t acc_shift = nAcc == 4u ? 2u : 1u;
     const uint32_t b_sub = (uint32_t)n_pad * 128u;
 
     extern __shared__ uint8_t smem_raw[];
@@ -433,10 +434,10 @@ stream_kernel(const uint8_t* __restrict__ table)
             for (int it = it0; it < it1 && ok && !*abort_flag; ++it, ++n) {
                 const ItemView v = view(it);
                 last_status = v.P->status;
-                const uint32_t ab = n % nAcc, lap = n / nAcc;
+                const uint32_t ab = n & (nAcc - 1u), lap = n >> acc_shift;      // nAcc is 2 or 4
                 bool have_acc = false;                    // this issuer has made sure the item's accumulator buffer is free
                 for (int st = 0; st < v.nst; ++st, ++t) {
-                    if ((int)(t % (uint32_t)nch) == me) {
+                    if ((int)(t & (uint32_t)(nch - 1)) == me) {                      // nch is 1, 2 or 4
                         if (!have_acc) {
                             if (!mbar_wait_parked(bar_tempty + 8 * ab, (lap & 1) ^ 1, abort_flag)) { ok = false; break; }
                             have_acc = true;
@@ -444,7 +445,7 @@ stream_kernel(const uint8_t* __restrict__ table)
                         if (!mbar_wait_parked(bar_fullB + 8 * sa, phA, abort_flag) || !mbar_wait_parked(bar_fullA + 8 * sa, phA, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         if (issuer) {
-                            const uint32_t chain = (uint32_t)st % (uint32_t)nch;
+                            const uint32_t chain = (uint32_t)st & (uint32_t)(nch - 1);
                             const uint32_t d_tmem = tmem_base + ab * acc_cols + chain * (uint32_t)n_pad;
                             const uint32_t a_t = tmem_base + a_base_col + sa * kAStageCols, b_lo = b_lo0 + sa * (b_bytes >> 4);
                             // a 32-code step is 8 columns of A and 32 bytes (two 16-byte units) of a B row; the first
@@ -553,8 +554,8 @@ stream_kernel(const uint8_t* __restrict__ table)
             const StreamProblem* P = vi.P;
             last_status = P->status;
             row_info(it + 1, scale_n, shift_n, m_n);
-            const uint32_t ab = n % nAcc;
-            if (!mbar_wait_parked_warp(bar_tfull + 8 * ab, (n / nAcc) & 1, abort_flag)) { alive = false; break; }
+            const uint32_t ab = n & (nAcc - 1u);
+            if (!mbar_wait_parked_warp(bar_tfull + 8 * ab, (n >> acc_shift) & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * acc_cols;
             const int N = P->N;
@@ -564,9 +565,11 @@ stream_kernel(const uint8_t* __restrict__ table)
             const int64_t ld = P->ld_out;
             const bool out_mn = P->out_mn != 0;
             // one value of this lane's row: undo the x16 of Fixed-4 rows, scale, store (and the raw sum if asked for)
+            // this lane's row: where its value of token nn goes
+            const int64_t o_row = out_mn ? (int64_t)m * ld : (int64_t)m, o_tok = out_mn ? 1 : ld;
             auto put = [&](int nn, uint32_t raw) {
                 const int a = (int)raw >> shift;
-                const int64_t o = out_mn ? (int64_t)m * ld + nn : (int64_t)nn * ld + m;
+                const int64_t o = o_row + (int64_t)nn * o_tok;
                 out[o] = __fmul_rn(__int2float_rn(a), scale);
                 if (acc) acc[o] = a;
             };
