@@ -678,3 +678,25 @@ def test_patch_matrix_rejects_bad_arguments():
         with pytest.raises(R.RmsmpError) as e:
             R.rmsmp_im2col_codes(*args)
         assert e.value.status == status
+
+
+# ---------------------------------------------------------------- resident weights expanded by the CTA itself
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,K,N,layout", [
+    (48, 192, 300, R.OUT_MN),       # duplicated rows (M <= 64), 64-byte k-blocks, [M][N] output
+    (100, 64, 515, R.OUT_NM),       # rows beyond M in the block, one short k-block
+    (128, 576, 77, R.OUT_NM),       # the largest resident stripe (72 KB expanded)
+    (64, 448, 1000, R.OUT_NM),      # 64-byte k-blocks with a last chunk of 64 codes
+])
+def test_linear_layer_without_workspace_on_resident_weights(M, K, N, layout):
+    """A layer of one row block whose expanded weights stay in shared memory is expanded once per CTA from the
+    packed codes (no workspace): every kind of row, both output layouts, with the raw sums."""
+    g = synth.rng(93, M + K + N)
+    W = synth.weights_normal(g, (M, K))
+    scheme, bits = _mixed_map(M, M + K, (50, 30, 20))
+    alpha = synth.alpha_rows(W)
+    act = g.integers(-8, 16, (N, K), dtype=np.int8)
+    layer, d_packed = Hn.pack_layer(W, scheme, bits, alpha)
+    y, acc = Hn.gemm(layer, d_packed, act, 0.125, R.VARIANT_TENSOR, out_layout=layout)
+    v_ref, ws = O.quantize_rows(W, scheme, bits, alpha)
+    _check_layer_outputs(y, acc, O.matmul(v_ref, act), ws, np.float32(0.125), alpha, scheme, bits)
