@@ -73,7 +73,7 @@ constexpr int kMaxTokens = 128;                                       // accumul
 constexpr int kRingMax = 12;
 constexpr int kStreamMaxK = 16384;                                    // reduction length up to which the fp32 sums of PoT tiles are exact
 constexpr int kLocalItems = 96;                                        // items of a CTA's list kept in shared memory
-constexpr int kStreamSmem = 232448 - 1024 - kLocalItems * 32;
+constexpr int kStreamSmem = 232448 - 1024 - kLocalItems * 16;
 constexpr uint32_t kPlanMagic = 0x53545247u;                          // "STRG"
 
 // One layer of the launch as the kernel sees it (device table, 128-byte aligned: it starts with
@@ -100,7 +100,10 @@ static_assert(sizeof(StreamProblem) % 128 == 0, "tensor maps stay 128-byte align
 
 // One tile: `rows` (1..128) consecutive packed rows of one kind, starting at row `row0` of their storage
 // region (4-bit or 8-bit) and at position `packed0` of the layer's permutation.
-struct StreamItem { int32_t prob, kind_rows, row0, packed0; };      // kind_rows = kind << 16 | rows
+struct StreamItem { int32_t prob, kind_rows, row0, packed0; };      // kind_rows = kind << 28 | k-blocks of the layer << 8 | rows
+__host__ __device__ inline int item_kind(int kr) { return (kr >> 28) & 3; }
+__host__ __device__ inline int item_nkb(int kr) { return (kr >> 8) & 0xFFFFF; }
+__host__ __device__ inline int item_rows(int kr) { return kr & 0xFF; }
 
 struct StreamHeader {               // first 128 bytes of the table
     uint32_t magic;
@@ -302,17 +305,16 @@ stream_kernel(const uint8_t* __restrict__ table)
     const uint32_t bar_tfull = sBar + 48 * kRingMax, bar_tempty = bar_tfull + 32;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    struct LocalItem { int4 a; int nkb, pad[3]; };        // the table's item (prob, kind << 16 | rows, row0, packed0) and its layer's k-blocks
-    __shared__ LocalItem s_items[kLocalItems];
+    __shared__ int4 s_items[kLocalItems];                 // the head of this CTA's list of items (prob, kind / k-blocks / rows, row0, packed0)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int it0 = __ldg(cta_first + blockIdx.x), it1 = __ldg(cta_first + blockIdx.x + 1);
     for (int i = threadIdx.x; i < min(it1 - it0, kLocalItems); i += kStreamThreads) {
-        const int4 a = __ldg(reinterpret_cast<const int4*>(items + it0 + i));
-        s_items[i].a = a;
-        s_items[i].nkb = probs[a.x].nkb;
+        s_items[i] = __ldg(reinterpret_cast<const int4*>(items + it0 + i));
     }
 
+    int pf_it = it0, pf_st = 0;                           // thread 0: where its early copies stopped (item, stage)
+    uint32_t pf_n = 0;                                    // ... and how many stages they were (at most one lap of the ring)
     if (threadIdx.x == 0) {
         for (int s = 0; s < kRingMax; ++s) {
             mbar_init(bar_fullA + 8 * s, kExpWarps / 2); // one arrival per expander warp of the set that has the stage
@@ -327,6 +329,23 @@ stream_kernel(const uint8_t* __restrict__ table)
         }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // This thread is also the producer of the packed codes: the first lap of the ring needs no wait, so its copies
+        // go out now, while the other warps are still setting up (tensor-memory allocation, the CTA-wide barrier).
+        while (pf_it < it1 && pf_n < (uint32_t)nS) {
+            const int4 a = __ldg(reinterpret_cast<const int4*>(items + pf_it));
+            const int kind = item_kind(a.y), nkb = item_nkb(a.y), bi = box_index(item_rows(a.y));
+            const int nst = (kind == kFixed8) ? nkb : (nkb + 1) >> 1;
+            const StreamProblem* P = probs + a.x;
+            const CUtensorMap* map = (kind == kFixed8) ? &P->q8[bi] : &P->q4[bi];
+            const uint32_t tx = (uint32_t)(128 >> bi) * 128u;
+            while (pf_st < nst && pf_n < (uint32_t)nS) {
+                const uint32_t fbar = bar_full + 8 * pf_n;
+                mbar_arrive_expect_tx(fbar, tx);
+                tma_load_2d(sRing + pf_n * stage_bytes, map, fbar, pf_st * 128, a.z);
+                ++pf_st; ++pf_n;
+            }
+            if (pf_st == nst) { ++pf_it; pf_st = 0; }
+        }
     }
     if (warp == kFirstMma) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem_base)) : "memory");
@@ -346,16 +365,11 @@ stream_kernel(const uint8_t* __restrict__ table)
     struct ItemView { const StreamProblem* P; int kind, rows, kbps, nst, nkb, row0, packed0; };
     auto view = [&](int it) -> ItemView {
         ItemView v;
-        int4 a; int nkb;
-        if (it - it0 < kLocalItems) {
-            a = s_items[it - it0].a; nkb = s_items[it - it0].nkb;
-        } else {
-            a = __ldg(reinterpret_cast<const int4*>(items + it));
-            nkb = probs[a.x].nkb;
-        }
+        const int4 a = (it - it0 < kLocalItems) ? s_items[it - it0] : __ldg(reinterpret_cast<const int4*>(items + it));
+        const int nkb = item_nkb(a.y);
         v.P = probs + a.x;
-        v.kind = a.y >> 16;
-        v.rows = a.y & 0xFFFF;
+        v.kind = item_kind(a.y);
+        v.rows = item_rows(a.y);
         v.row0 = a.z; v.packed0 = a.w;
         v.nkb = nkb;
         v.kbps = (v.kind == kFixed8) ? 1 : 2;
@@ -366,9 +380,9 @@ stream_kernel(const uint8_t* __restrict__ table)
     if (warp == 0) {
         // ---------------------------------------------------------- producer of the packed codes (one lane)
         if (lane == 0) {
-            uint32_t sr = 0, phR = 0;
+            uint32_t sr = pf_n == (uint32_t)nS ? 0u : pf_n, phR = pf_n == (uint32_t)nS ? 1u : 0u;
             bool ok = true;
-            for (int it = it0; it < it1 && ok; ++it) {
+            for (int it = pf_it; it < it1 && ok; ++it) {
                 const ItemView v = view(it);
                 last_status = v.P->status;
                 const int bi = box_index(v.rows);
@@ -380,7 +394,7 @@ stream_kernel(const uint8_t* __restrict__ table)
                     tensormap_prefetch((nv.kind == kFixed8) ? &nv.P->q8[nb] : &nv.P->q4[nb]);
                 }
                 const uint32_t tx = (uint32_t)(128 >> bi) * 128u;
-                for (int st = 0; st < v.nst; ++st) {
+                for (int st = (it == pf_it) ? pf_st : 0; st < v.nst; ++st) {
                     if (!mbar_wait_parked(bar_empty + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
                     const uint32_t fbar = bar_full + 8 * sr;
                     mbar_arrive_expect_tx(fbar, tx);
@@ -671,6 +685,7 @@ bool stream_supported(const Problem& p)
     if (p.pix_pitch % 16 != 0 || (reinterpret_cast<uintptr_t>(p.act) & 15) != 0) return false;
     // PoT tiles are summed in fp32 in units of 1/4: exact while 64 * 16 * K <= 2^24
     if (p.nP > 0 && p.Kp > kStreamMaxK) return false;
+    if (p.Kp / 128 >= (1 << 20)) return false;                  // the k-block count travels in 20 bits of an item's word
     return tensor_map_encoder() != nullptr;
 }
 
@@ -804,7 +819,7 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
                 // the height of its box; an item's start-up and output about 3/4 of a full stage
                 static const int kind_weight[3] = {111, 100, 79};
                 const int64_t cost = (int64_t)nst * kind_weight[k] * (64 + (64 >> box_index(rows))) + 9600;
-                cand.push_back({cost, {i, (k << 16) | rows, region_row0[k] + r, perm0[k] + r}});
+                cand.push_back({cost, {i, (k << 28) | (nkb << 8) | rows, region_row0[k] + r, perm0[k] + r}});
             }
     }
     std::stable_sort(cand.begin(), cand.end(), [](const Cand& a, const Cand& b) { return a.cost > b.cost; });
