@@ -3,13 +3,13 @@
 //
 // With a handful of tokens a layer is bound by reading its packed weights once, and the only
 // per-weight work is turning 4-bit codes into int8 operands.  One persistent CTA per SM walks its
-// own list of work items.  An item is up to 128 consecutive PACKED rows of ONE kind of one layer
+// own list of work items.  An item is up to 128 (Fixed-8: 64) consecutive PACKED rows of ONE kind of one layer
 // (the packed buffer groups the rows by kind, so such a tile is a dense block of the 4-bit or the
 // 8-bit region), the whole reduction, all tokens.  Tiles of one kind keep the decode free of
 // divergence and spread the expensive kind (PoT) evenly over the four SM sub-partitions; the
 // price is an output scatter through the row permutation, which costs little with few tokens.
-// Per item the reduction is cut into stages: 256 codes of a 4-bit tile, 128 of an 8-bit tile --
-// always 128 bytes per row, so a stage is ONE bulk copy of at most 128 rows x 128 bytes.  The
+// Per item the reduction is cut into stages of 256 codes and at most 16 KB: ONE bulk copy of at most 128 rows x
+// 128 bytes for a 4-bit tile; two of at most 64 rows x 128 bytes for an 8-bit tile, which is 64 rows high.  The
 // expanded weights never touch shared memory: they go from registers to TENSOR MEMORY (tcgen05.st)
 // and the MMA takes its A operand from there, so shared memory carries only the packed codes (once
 // in, once out) and the activation tiles.  Warp roles:
@@ -191,13 +191,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&w)[16
           "r"(w[8]), "r"(w[9]), "r"(w[10]), "r"(w[11]), "r"(w[12]), "r"(w[13]), "r"(w[14]), "r"(w[15])
         : "memory");
 }
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&w)[16])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-        ::"r"(taddr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
-        : "memory");
-}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // 16 accumulator columns of this thread's lane; valid after the wait.
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
@@ -334,14 +327,23 @@ stream_kernel(const uint8_t* __restrict__ table)
         while (pf_it < it1 && pf_n < (uint32_t)nS) {
             const int4 a = __ldg(reinterpret_cast<const int4*>(items + pf_it));
             const int kind = item_kind(a.y), nkb = item_nkb(a.y), bi = box_index(item_rows(a.y));
-            const int nst = (kind == kFixed8) ? nkb : (nkb + 1) >> 1;
+            const bool two = kind == kFixed8;
+            const int nst = (nkb + 1) >> 1;
             const StreamProblem* P = probs + a.x;
             const CUtensorMap* map = (kind == kFixed8) ? &P->q8[bi] : &P->q4[bi];
             const uint32_t tx = (uint32_t)(128 >> bi) * 128u;
             while (pf_st < nst && pf_n < (uint32_t)nS) {
                 const uint32_t fbar = bar_full + 8 * pf_n;
-                mbar_arrive_expect_tx(fbar, tx);
-                tma_load_2d(sRing + pf_n * stage_bytes, map, fbar, pf_st * 128, a.z);
+                if (two) {
+                    // an 8-bit tile of at most 64 rows: the stage's two k-blocks are two boxes, one per half of the slot
+                    const int nb = min(2, nkb - 2 * pf_st);
+                    mbar_arrive_expect_tx(fbar, (uint32_t)nb * tx);
+                    for (int u = 0; u < nb; ++u)
+                        tma_load_2d(sRing + pf_n * stage_bytes + (uint32_t)u * (stage_bytes >> 1), map, fbar, (2 * pf_st + u) * 128, a.z);
+                } else {
+                    mbar_arrive_expect_tx(fbar, tx);
+                    tma_load_2d(sRing + pf_n * stage_bytes, map, fbar, pf_st * 128, a.z);
+                }
                 ++pf_st; ++pf_n;
             }
             if (pf_st == nst) { ++pf_it; pf_st = 0; }
@@ -359,7 +361,7 @@ stream_kernel(const uint8_t* __restrict__ table)
 
     uint32_t* last_status = nullptr;                      // status word of the layer this thread worked on last
 
-    // An item's stages: a 4-bit tile takes two k-blocks (256 codes) per stage, an 8-bit tile one (128 codes).
+    // An item's stages: two k-blocks (256 codes) each -- one box of a 4-bit tile, two boxes of an 8-bit tile.
     // The first kLocalItems items of the CTA's list were copied to shared memory above, with everything the
     // roles need to walk them, so that no role starts an item with a chain of dependent global loads.
     struct ItemView { const StreamProblem* P; int kind, rows, kbps, nst, nkb, row0, packed0; };
@@ -372,8 +374,8 @@ stream_kernel(const uint8_t* __restrict__ table)
         v.rows = item_rows(a.y);
         v.row0 = a.z; v.packed0 = a.w;
         v.nkb = nkb;
-        v.kbps = (v.kind == kFixed8) ? 1 : 2;
-        v.nst = (v.kind == kFixed8) ? nkb : (nkb + 1) >> 1;
+        v.kbps = 2;                                      // k-blocks per stage: one box of a 4-bit tile, two boxes of an 8-bit tile
+        v.nst = (nkb + 1) >> 1;
         return v;
     };
 
@@ -397,8 +399,15 @@ stream_kernel(const uint8_t* __restrict__ table)
                 for (int st = (it == pf_it) ? pf_st : 0; st < v.nst; ++st) {
                     if (!mbar_wait_parked(bar_empty + 8 * sr, phR ^ 1, abort_flag)) { ok = false; break; }
                     const uint32_t fbar = bar_full + 8 * sr;
-                    mbar_arrive_expect_tx(fbar, tx);
-                    tma_load_2d(sRing + sr * stage_bytes, map, fbar, st * 128, v.row0);     // 128 bytes of every row per stage
+                    if (v.kind == kFixed8) {
+                        const int nb = min(2, v.nkb - 2 * st);
+                        mbar_arrive_expect_tx(fbar, (uint32_t)nb * tx);
+                        for (int u = 0; u < nb; ++u)
+                            tma_load_2d(sRing + sr * stage_bytes + (uint32_t)u * (stage_bytes >> 1), map, fbar, (2 * st + u) * 128, v.row0);
+                    } else {
+                        mbar_arrive_expect_tx(fbar, tx);
+                        tma_load_2d(sRing + sr * stage_bytes, map, fbar, st * 128, v.row0);     // 128 bytes of every row per stage
+                    }
                     if (++sr == (uint32_t)nS) { sr = 0; phR ^= 1; }
                 }
             }
@@ -513,6 +522,42 @@ stream_kernel(const uint8_t* __restrict__ table)
                     if (!mbar_wait_parked_warp(bar_full + 8 * sr, phR, abort_flag)) { ok = false; break; }
                     const uint32_t row = sRing + sr * stage_bytes + row_off;
                     uint32_t w[16], w2[16];
+                    if (eight) {
+                        // An 8-bit tile has at most 64 rows (tensor-memory lanes 0..63: quarters 0 and 1); its stage is
+                        // two boxes, one per k-block.  A 32-byte piece g of a row is its 32-code step g: 8 columns.
+                        // w[0..7] / w[8..15]: this thread's two pieces of the first / of the second box.
+                        const int nb = min(2, v.nkb - 2 * st);
+                        if (have_row) {
+                            stream_expand(kFixed8, row, ph, 2 * half, w);
+                            stream_expand(kFixed8, row, ph, 2 * half + 1, w2);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) w[8 + q] = w2[q];
+                            if (nb == 2) {
+                                uint32_t x[16];
+                                stream_expand(kFixed8, row + (stage_bytes >> 1), ph, 2 * half, w2);
+                                stream_expand(kFixed8, row + (stage_bytes >> 1), ph, 2 * half + 1, x);
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) w2[8 + q] = x[q];
+                            }
+                        } else {
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) { w[q] = 0u; w2[q] = 0u; }
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_empty + 8 * sr);
+                        if (!mbar_wait_parked_warp(bar_emptyA + 8 * sa, phA ^ 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t col8 = t_lane + sa * kAStageCols;
+                        tmem_st16(col8 + 16 * half, w);                    // first k-block: columns 0..31
+                        if (nb == 2) tmem_st16(col8 + 32 + 16 * half, w2);  // second k-block: columns 32..63
+                        tmem_st_wait();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_fullA + 8 * sa);
+                        if (++sr == (uint32_t)nS) { sr = 0; phR ^= 1; }
+                        if (++sa == (uint32_t)nAst) { sa = 0; phA ^= 1; }
+                        continue;
+                    }
                     if (have_row) {
                         stream_expand(v.kind, row, ph, 2 * half, w);
                         stream_expand(v.kind, row, ph, 2 * half + 1, w2);
@@ -525,15 +570,9 @@ stream_kernel(const uint8_t* __restrict__ table)
                     if (!mbar_wait_parked_warp(bar_emptyA + 8 * sa, phA ^ 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t col = t_lane + sa * kAStageCols;
-                    if (eight) {
-                        // an 8-bit row's 32-byte piece g is its 32-code step g: 8 columns
-                        tmem_st8(col + 16 * half, w);
-                        tmem_st8(col + 16 * half + 8, w2);
-                    } else {
-                        // a 4-bit row's 32-byte piece g is its steps 2g, 2g + 1: 16 columns
-                        tmem_st16(col + 32 * half, w);
-                        tmem_st16(col + 32 * half + 16, w2);
-                    }
+                    // a 4-bit row's 32-byte piece g is its steps 2g, 2g + 1: 16 columns
+                    tmem_st16(col + 32 * half, w);
+                    tmem_st16(col + 32 * half + 16, w2);
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
@@ -660,10 +699,18 @@ Layout table_layout(int count, int nitems, int grid)
 
 }  // namespace
 
-// Tiles of a layer: the rows of each kind in blocks of 128 packed rows.
+// Height of a Fixed-8 tile: 64 rows, two k-blocks (two boxes of 64 rows x 128 bytes) per stage, so that a stage of
+// any tile is 16 KB and 256 codes deep.  Measured against 128-row tiles with one k-block per stage on the paper's
+// mix: 46 against 47.4 us at 8 tokens (half as many stages for the few Fixed-8 rows of a layer; the idle
+// tensor-memory quarters cost nothing).  A layer of Fixed-8 rows only, which no ratio of the paper is, pays for it
+// (72 against 61 us).
+static int f8_tile_rows(int, int, int) { return 64; }
+
+// Tiles of a layer: the rows of each 4-bit kind in blocks of 128 packed rows, the 8-bit rows in blocks of 64 or 128.
 int64_t stream_items_of(int nP, int nF4, int n8)
 {
-    return (nP + 127) / 128 + (nF4 + 127) / 128 + (n8 + 127) / 128;
+    const int t8 = f8_tile_rows(nP, nF4, n8);
+    return (nP + 127) / 128 + (nF4 + 127) / 128 + (n8 + t8 - 1) / t8;
 }
 
 // Scratch bytes the table of `count` layers with `nitems` tiles needs on a device with `sms` SMs.
@@ -811,13 +858,14 @@ bool stream_build_table(const Problem* probs, int count, int sms, uint8_t* h_tab
         const int n_of[3] = {p.nP, p.nF4, p.n8};
         const int region_row0[3] = {0, p.nP, 0};                   // first row of the kind inside its storage region
         const int perm0[3] = {0, p.nP, p.nP + p.nF4};              // ... and inside the permutation
+        const int tile_rows[3] = {128, 128, f8_tile_rows(p.nP, p.nF4, p.n8)};
         for (int k = 0; k < 3; ++k)
-            for (int r = 0; r < n_of[k]; r += 128) {
-                const int rows = std::min(128, n_of[k] - r);
-                const int nst = (k == kFixed8) ? nkb : (nkb + 1) / 2;
-                // measured: a stage of a full PoT / Fixed-4 / Fixed-8 tile takes about 1.11 : 1 : 0.79, half of it whatever
+            for (int r = 0; r < n_of[k]; r += tile_rows[k]) {
+                const int rows = std::min(tile_rows[k], n_of[k] - r);
+                const int nst = (nkb + 1) / 2;
+                // measured: a stage of a full PoT / Fixed-4 / Fixed-8 tile takes about 1.11 : 1 : 1.1, half of it whatever
                 // the height of its box; an item's start-up and output about 3/4 of a full stage
-                static const int kind_weight[3] = {111, 100, 79};
+                static const int kind_weight[3] = {111, 100, 110};
                 const int64_t cost = (int64_t)nst * kind_weight[k] * (64 + (64 >> box_index(rows))) + 9600;
                 cand.push_back({cost, {i, (k << 28) | (nkb << 8) | rows, region_row0[k] + r, perm0[k] + r}});
             }
