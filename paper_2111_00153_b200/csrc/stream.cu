@@ -450,7 +450,7 @@ stream_kernel(const uint8_t* __restrict__ table)
         const int me = warp - kFirstMma;
         if (me < nch) {
             const bool issuer = (lane == 0);
-            uint32_t sa = 0, phA = 0, n = 0, t = 0;
+            uint32_t sa = (uint32_t)me, phA = 0, n = 0, t = 0;        // t: stages of the items before this one
             const uint64_t desc_b0 = smem_desc_kmajor(sB, 128);
             const uint32_t b_lo0 = (uint32_t)desc_b0, desc_hi = (uint32_t)(desc_b0 >> 32);
             bool ok = true;
@@ -459,8 +459,10 @@ stream_kernel(const uint8_t* __restrict__ table)
                 last_status = v.P->status;
                 const uint32_t ab = n & (nAcc - 1u), lap = n >> acc_shift;      // nAcc is 2 or 4
                 bool have_acc = false;                    // this issuer has made sure the item's accumulator buffer is free
-                for (int st = 0; st < v.nst; ++st, ++t) {
-                    if ((int)(t & (uint32_t)(nch - 1)) == me) {                      // nch is 1, 2 or 4
+                // its own stages only: those whose index over the whole list is me modulo nch (1, 2 or 4); the A stage
+                // advances by nch with them (nch <= nAst)
+                for (int st = (int)(((uint32_t)me - t) & (uint32_t)(nch - 1)); st < v.nst; st += nch) {
+                    {
                         if (!have_acc) {
                             if (!mbar_wait_parked(bar_tempty + 8 * ab, (lap & 1) ^ 1, abort_flag)) { ok = false; break; }
                             have_acc = true;
@@ -488,8 +490,10 @@ stream_kernel(const uint8_t* __restrict__ table)
                             mma_commit(bar_emptyA + 8 * sa);
                         }
                     }
-                    if (++sa == (uint32_t)nAst) { sa = 0; phA ^= 1; }
+                    sa += (uint32_t)nch;
+                    if (sa >= (uint32_t)nAst) { sa -= (uint32_t)nAst; phA ^= 1; }
                 }
+                t += (uint32_t)v.nst;
                 if (!ok) break;
                 // Every issuer reports once per item, whether or not a stage of it was its own.  An issuer without
                 // stages in short items can be items ahead of the others: before it reports on this buffer again
@@ -509,16 +513,22 @@ stream_kernel(const uint8_t* __restrict__ table)
         const int slot = quarter * 32 + lane;            // the thread's row of every tile
         const uint32_t row_off = (uint32_t)slot * 128u, ph = (uint32_t)(slot & 7);
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + a_base_col;
-        uint32_t t = 0;                                  // stages this CTA has been through
-        uint32_t sr = 0, phR = 0, sa = 0, phA = 0;       // ring positions of stage t (advanced for every stage, taken or not)
+        uint32_t t = 0;                                  // stages of the items before the current one
+        // ring positions of the set's next stage: its stages are every other one of the CTA's list, so both rings
+        // advance by two with them (nS >= 2, nAst even)
+        uint32_t sr = (uint32_t)set, phR = 0, sa = (uint32_t)set, phA = 0;
+        auto advance = [&]() {
+            sr += 2u; if (sr >= (uint32_t)nS) { sr -= (uint32_t)nS; phR ^= 1; }
+            sa += 2u; if (sa >= (uint32_t)nAst) { sa -= (uint32_t)nAst; phA ^= 1; }
+        };
         bool ok = true;
         for (int it = it0; it < it1 && ok; ++it) {
             const ItemView v = view(it);
             last_status = v.P->status;
             const bool have_row = slot < v.rows;         // lanes beyond the tile's rows hand zeros to the MMA
             const bool eight = v.kind == kFixed8;
-            for (int st = 0; st < v.nst; ++st, ++t) {
-                if ((int)(t & 1u) == set) {
+            for (int st = (int)(((uint32_t)set - t) & 1u); st < v.nst; st += 2) {
+                {
                     if (!mbar_wait_parked_warp(bar_full + 8 * sr, phR, abort_flag)) { ok = false; break; }
                     const uint32_t row = sRing + sr * stage_bytes + row_off;
                     uint32_t w[16], w2[16];
@@ -554,8 +564,7 @@ stream_kernel(const uint8_t* __restrict__ table)
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_fullA + 8 * sa);
-                        if (++sr == (uint32_t)nS) { sr = 0; phR ^= 1; }
-                        if (++sa == (uint32_t)nAst) { sa = 0; phA ^= 1; }
+                        advance();
                         continue;
                     }
                     if (have_row) {
@@ -578,9 +587,9 @@ stream_kernel(const uint8_t* __restrict__ table)
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_fullA + 8 * sa);
                 }
-                if (++sr == (uint32_t)nS) { sr = 0; phR ^= 1; }
-                if (++sa == (uint32_t)nAst) { sa = 0; phA ^= 1; }
+                advance();
             }
+            t += (uint32_t)v.nst;
         }
     } else {
         // ---------------------------------------------------------- epilogue
