@@ -164,7 +164,8 @@ __device__ __forceinline__ uint32_t e4m3x4_of_s8x4(uint32_t w)
 // 32-byte piece `g` (0..3) of this thread's 128-byte raw row, expanded to 16 words of int8 values:
 // a 4-bit row: its 32-code steps 2g and 2g + 1 (w[0..7], w[8..15]); an 8-bit row: its step g (w[0..7]; the
 // rest is not used).  `row` = shared-memory address of the row, ph = its swizzle phase (row & 7).
-__device__ __forceinline__ void stream_expand(int kind, uint32_t row, uint32_t ph, int g, uint32_t (&w)[16])
+template <int kind>
+__device__ __forceinline__ void stream_expand(uint32_t row, uint32_t ph, int g, uint32_t (&w)[16])
 {
     uint4 c0, c1;
     const uint32_t a0 = row + (((uint32_t)(2 * g) ^ ph) << 4);
@@ -538,14 +539,14 @@ stream_kernel(const uint8_t* __restrict__ table)
                         // w[0..7] / w[8..15]: this thread's two pieces of the first / of the second box.
                         const int nb = min(2, v.nkb - 2 * st);
                         if (have_row) {
-                            stream_expand(kFixed8, row, ph, 2 * half, w);
-                            stream_expand(kFixed8, row, ph, 2 * half + 1, w2);
+                            stream_expand<kFixed8>(row, ph, 2 * half, w);
+                            stream_expand<kFixed8>(row, ph, 2 * half + 1, w2);
 #pragma unroll
                             for (int q = 0; q < 8; ++q) w[8 + q] = w2[q];
                             if (nb == 2) {
                                 uint32_t x[16];
-                                stream_expand(kFixed8, row + (stage_bytes >> 1), ph, 2 * half, w2);
-                                stream_expand(kFixed8, row + (stage_bytes >> 1), ph, 2 * half + 1, x);
+                                stream_expand<kFixed8>(row + (stage_bytes >> 1), ph, 2 * half, w2);
+                                stream_expand<kFixed8>(row + (stage_bytes >> 1), ph, 2 * half + 1, x);
 #pragma unroll
                                 for (int q = 0; q < 8; ++q) w2[8 + q] = x[q];
                             }
@@ -567,9 +568,12 @@ stream_kernel(const uint8_t* __restrict__ table)
                         advance();
                         continue;
                     }
-                    if (have_row) {
-                        stream_expand(v.kind, row, ph, 2 * half, w);
-                        stream_expand(v.kind, row, ph, 2 * half + 1, w2);
+                    if (have_row && v.kind == kPoT4) {
+                        stream_expand<kPoT4>(row, ph, 2 * half, w);
+                        stream_expand<kPoT4>(row, ph, 2 * half + 1, w2);
+                    } else if (have_row) {
+                        stream_expand<kFixed4>(row, ph, 2 * half, w);
+                        stream_expand<kFixed4>(row, ph, 2 * half + 1, w2);
                     } else {
 #pragma unroll
                         for (int q = 0; q < 16; ++q) { w[q] = 0u; w2[q] = 0u; }
